@@ -1,0 +1,34 @@
+"""Globally-randomized blockwise sparsifier (GRBS), Definition 2 (oracle side).
+
+Test infrastructure only.  The flat vector of d elements is cut into
+B = ceil(d / block_size) contiguous blocks (the last one may be short).  Every
+worker derives the same selection from a shared seed, so the mask is a function
+of (seed, step t, which compressor, block b) alone.  Reading taken where the
+paper gives no sampling procedure: each block is selected independently with
+probability 1/R, which makes C(v) = v * mask a 1/R-approximate compressor in
+expectation exactly as Definition 2 states.
+
+Draw: word 0 of Philox4x32-10 with key = (seed low 32 bits, seed high 32 bits)
+and counter = (b, t low 32 bits, t high 32 bits, stream), stream 0 for the
+per-step compressor of the update, 1 for the error-reset compressor.  Block b
+is selected iff  word0 * R < 2**32  (R = 1 selects everything).
+"""
+import numpy as np
+from .philox import philox4x32_10
+
+STREAM_GRAD = 0    # compressor applied to the update p every step (Algorithm 2 line 6)
+STREAM_RESET = 1   # compressor applied to the error e every H steps (Algorithm 2 line 11)
+
+
+def n_blocks(d, block_size):
+    return (int(d) + int(block_size) - 1) // int(block_size)
+
+
+def grbs_mask(seed, t, stream, B, R, block_begin=0):
+    """uint8[B] selection flags of blocks block_begin .. block_begin+B-1 at step t."""
+    seed = int(seed) & 0xFFFFFFFFFFFFFFFF
+    t = int(t) & 0xFFFFFFFFFFFFFFFF
+    b = np.arange(block_begin, block_begin + B, dtype=np.uint64)
+    word0 = philox4x32_10(seed & 0xFFFFFFFF, seed >> 32,
+                          b, t & 0xFFFFFFFF, t >> 32, int(stream))[0]
+    return (word0.astype(np.uint64) * np.uint64(R) < np.uint64(1 << 32)).astype(np.uint8)
