@@ -1,0 +1,325 @@
+#!/usr/bin/env python
+"""Benchmark of the CSER / M-CSER optimizer step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
+
+One "step" = one pass of the whole hot path (GRBS mask kernel + fused step kernel)
+over one [n, d] batch of synthetic gradients.  The headline workload is the
+WRN-40-8-sized configuration (d = 35,748,708, n = 8, R1 = R2 = 32, H = 8, beta = 0.9).
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank owns one column slab
+of that size with global block ids and no data is exchanged ("weak" scaling).
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "cser_steps_per_sec"
+UNIT = "steps/s"
+PEAK_NOMINAL_GBS = 8000.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused step kernel,
+# from the ncu capture summarised under profiles/ (None until captured).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+
+
+def algorithmic_bytes(w, frac_e_touched):
+    """Bytes one step must move: g read; x, (m) read+write; e read+write where touched."""
+    per = 4 + 8 + (8 if w.beta != 0 else 0) + 8 * frac_e_touched
+    return w.n_workers * w.d * per
+
+
+def expected_e_fraction(w, is_reset):
+    f = 1.0 - 1.0 / w.R1
+    if is_reset:
+        f = 1.0 - (1.0 / w.R1) * (1.0 - 1.0 / w.R2)
+    return f
+
+
+def mean_algorithmic_bytes(w, t_first, k):
+    tot = 0.0
+    for t in range(t_first, t_first + k):
+        tot += algorithmic_bytes(w, expected_e_fraction(w, t % w.H == 0))
+    return tot / k
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML (read-only) while a region runs."""
+
+    def __init__(self, device_index):
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self.nv, self.h = pynvml, pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception as ex:  # NVML not reachable: report that instead of numbers
+            self.nv, self.err = None, repr(ex)
+
+    def _poll(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20,
+                 "hw_thermal_slowdown": 0x40, "hw_power_brake": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.004)
+
+    def __enter__(self):
+        if self.nv:
+            self._thr = threading.Thread(target=self._poll, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thr:
+            self._thr.join()
+
+    def summary(self):
+        if not self.nv:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvml unavailable: " + self.err]}
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def oracle_sample_rate(w, target_seconds=15.0, sample_cols=1 << 18):
+    """Time the CPU oracle, as it stands, on a contiguous slab of whole blocks of workload w.
+    Returns (full-vector steps/s equivalent, description, threads used)."""
+    import numpy as np
+    import torch
+    from oracle import CSEROracle
+    from paper_2007_13221_b200 import synth
+    cols_n = min(w.d, sample_cols // w.block_size * w.block_size)
+    ws = w.scaled(cols_n)
+    ref = CSEROracle(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
+                     dtype=np.float64, cols=np.arange(cols_n))
+    ref.set_x0(synth.x0(ws, "cpu").numpy())
+    grads = [synth.gradients(ws, t, "cpu").numpy() for t in range(1, 5)]
+    ref.step(grads[0])                                    # warm-up (page faults, imports)
+    n_steps, t0 = 0, time.perf_counter()
+    while True:
+        ref.step(grads[n_steps % len(grads)])
+        n_steps += 1
+        el = time.perf_counter() - t0
+        if el >= target_seconds or n_steps >= 400:
+            break
+    rate = n_steps / el * (cols_n / w.d)
+    desc = (f"{n_steps} oracle steps (float64 NumPy) on the first {cols_n} of {w.d} columns x {w.n_workers} "
+            f"workers of {w.name}; rate scaled by {cols_n}/{w.d} to the full vector")
+    return rate, desc, 1, el
+
+
+def run_reference(args, w):
+    """--impl reference: the oracle, timed on the host cores, same metric and workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step_budget = 2.0
+    rates = []
+    t_all0 = time.perf_counter()
+    for k in range(args.warmup + args.steps):
+        rate, desc, cores, _ = oracle_sample_rate(w, target_seconds=per_step_budget, sample_cols=1 << 17)
+        if k >= args.warmup:
+            rates.append(rate)
+        if time.perf_counter() - t_all0 > 150:
+            break
+    value = len(rates) / sum(1.0 / r for r in rates)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / value, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "d": w.d, "n_workers": w.n_workers, "block_size": w.block_size,
+                   "R1": w.R1, "R2": w.R2, "H": w.H, "eta": w.eta, "beta": w.beta},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": "each timed step = " + desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--config", type=int, default=2, help="workload 1..5 (2 = headline)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--ring", type=int, default=0, help="distinct gradient buffers cycled through")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    from paper_2007_13221_b200 import synth
+    w = synth.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2007_13221_b200 import binding as b
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    import __graft_entry__
+    if rank == 0:
+        __graft_entry__.build()
+    if world > 1:
+        dist.barrier()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # each rank owns one slab of the workload's size, with global block ids
+    opt = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
+                 block_begin=rank * w.n_blocks)
+    opt.set_x0(synth.x0(w, dev))
+    g_bytes = w.n_workers * w.d * 4
+    ring_n = args.ring or max(2, min(4, int(6e9 // g_bytes)))
+    ring = [synth.gradients(w, 1 + k, dev) for k in range(ring_n)]
+    torch.cuda.synchronize()
+
+    stream = torch.cuda.current_stream()
+    K, W = args.steps, args.warmup
+    for k in range(W):
+        opt.step(ring[k % ring_n])
+    barrier()
+    launches0 = b.cser_launch_count(opt.h)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_first = opt.t + 1
+    with ClockSampler(local) as clocks:
+        ev0.record(stream)
+        for k in range(K):
+            opt.step(ring[k % ring_n])
+        ev1.record(stream)
+        barrier()
+    total_ms = ev0.elapsed_time(ev1)
+    launches = b.cser_launch_count(opt.h) - launches0
+    if world > 1:
+        tt = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / K
+    value = world * K / (total_ms * 1e-3)
+    alg_bytes = mean_algorithmic_bytes(w, t_first, K)
+
+    # per-kernel durations of the fused step kernel (CUDA events on the launching stream)
+    b.cser_set_timing(opt.h, True)
+    k_ms, k_bytes, mask_ms = [], [], []
+    n_prof = min(K, 4 * w.H if w.H > 1 else 16)
+    for k in range(n_prof):
+        opt.step(ring[k % ring_n])
+        a_ms, s_ms = b.cser_last_kernel_ms(opt.h)
+        mask_ms.append(a_ms), k_ms.append(s_ms)
+        k_bytes.append(algorithmic_bytes(w, expected_e_fraction(w, opt.t % w.H == 0)))
+    b.cser_set_timing(opt.h, False)
+    peak, peak_src = measured_peaks()
+    achieved = sum(k_bytes) / (sum(k_ms) * 1e-3) / 1e9
+    roofline = {
+        "bound": "hbm", "kernel": "cser_step_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "frac": achieved / peak, "peak_source": peak_src, "frac_of_nominal_8TBs": achieved / PEAK_NOMINAL_GBS,
+        "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(w.name),
+        "algorithmic_bytes_per_launch": sum(k_bytes) / len(k_bytes),
+        "kernel_ms_avg": sum(k_ms) / len(k_ms), "mask_kernel_ms_avg": sum(mask_ms) / len(mask_ms),
+        "launches_timed": len(k_ms),
+    }
+
+    # end to end: gradients start in pinned host memory every step; a result is read back
+    e2e = None
+    if not args.no_e2e:
+        host_ring = [torch.empty((w.n_workers, w.d), dtype=torch.float32).pin_memory() for _ in range(2)]
+        for hb, gb in zip(host_ring, ring):
+            hb.copy_(gb)
+        mask_host = torch.empty(w.n_blocks, dtype=torch.uint8).pin_memory()
+        ke = max(3, min(K, 12))
+        for k in range(2):
+            opt.step_host(host_ring[k % 2])
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for k in range(ke):
+            opt.step_host(host_ring[k % 2])
+            b.cser_read_state(opt.h, b.STATE_MASK_G, mask_host)
+            stream.synchronize()                      # the caller consumes the result every step
+            _ = opt.t
+        e1.record(stream)
+        barrier()
+        e_ms = e0.elapsed_time(e1)
+        if world > 1:
+            tt = torch.tensor([e_ms], device=dev)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e_ms = float(tt.item())
+        e2e = {"value": world * ke / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": g_bytes,
+               "d2h_bytes_per_step": w.n_blocks + 8, "steps": ke,
+               "note": "cser_step_host from pinned host gradients + read-back of the step's mask and t"}
+        del host_ring
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        rate, desc, cores, _ = oracle_sample_rate(w)
+        cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "d": w.d, "n_workers": w.n_workers, "block_size": w.block_size,
+                       "R1": w.R1, "R2": w.R2, "H": w.H, "eta": w.eta, "beta": w.beta,
+                       "parallelism": f"column slabs x{world}, no collective",
+                       "l2": f"inputs larger than L2: {alg_bytes / 1e9:.2f} GB touched per step, "
+                             f"{ring_n} gradient buffers cycled"},
+            "hbm_gbs_step": alg_bytes / (ms_per_step * 1e-3) / 1e9 * 1.0,
+            "hbm_frac_of_8TBs": alg_bytes / (ms_per_step * 1e-3) / 1e9 / PEAK_NOMINAL_GBS,
+            "algorithmic_bytes_per_step": alg_bytes,
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+            "gpu_launches": launches, "clocks": clocks.summary(),
+        }
+        print(json.dumps(line))
+    opt.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,178 @@
+/*
+ * cser.h - C ABI of the B200 (sm_100a) CSER / M-CSER optimizer-step library.
+ *
+ * What it computes.  n simulated workers each hold a local model x_i, a local
+ * error e_i and (with momentum) a local momentum m_i, all vectors of d fp32
+ * elements, stored as row-major [n, d] arrays in one GPU's memory.  One call of
+ * cser_step() performs one iteration t of "CSER" (Algorithm 2) or, when beta != 0,
+ * of "M-CSER, implementation I" (Algorithm 4) of arXiv 2007.13221 for all workers:
+ *
+ *   1. Get_p (Appendix A.4):    m_i <- beta*m_i + g_i ;  p_i <- eta*(beta*m_i + g_i)
+ *                               (beta == 0:  p_i <- eta*g_i)
+ *   2. PSync(p, C) (Algorithm 3) with the GRBS compressor of Definition 2:
+ *        selected blocks:    x_i <- x_i - mean_k p_k        (e_i unchanged)
+ *        unselected blocks:  x_i <- x_i - p_i ;  e_i <- e_i - p_i
+ *   3. if t mod H == 0, error reset (Algorithm 2 lines 11-12) with a second,
+ *      independently drawn GRBS mask, on its selected blocks only:
+ *        x_i <- (x_i - e_i) + mean_k e_k ;  e_i <- 0
+ *
+ * The mean over the worker axis is what a deployment would do with an allreduce.
+ *
+ * Naming.  R1 is the compression ratio of the compressor applied to the update
+ * every step (the paper's Algorithm 2 calls it C_2); R2 is the ratio of the
+ * compressor applied to the error every H steps (the paper's C_1).
+ *
+ * GRBS mask (Definition 2).  The vector is cut into B = ceil(d / block_size)
+ * contiguous blocks.  Block b is selected at step t for compressor s (0 = update,
+ * 1 = reset) iff  word0 * R < 2^32, where word0 is the first output word of
+ * Philox4x32-10 with key = (seed & 0xffffffff, seed >> 32) and counter =
+ * (b, t & 0xffffffff, t >> 32, s).  R = 1 selects every block; for any R each
+ * block is selected independently with probability ceil(2^32/R)/2^32 (= 1/R for
+ * powers of two), so the compressor is 1/R-approximate in expectation.
+ *
+ * Arithmetic.  fp32, round-to-nearest, no fused multiply-add, no flush-to-zero.
+ * Order: t1 = beta*m; m' = t1+g; t2 = beta*m'; t3 = t2+g; p = eta*t3.  Sums over
+ * workers run in ascending worker order starting from worker 0's value; the mean
+ * is sum / (float)n.  The reset computes (x - e) first, then adds the mean.
+ *
+ * Conventions.  t is 0 after cser_create / cser_set_x0; the first cser_step is
+ * t = 1; resets happen at t = H, 2H, ...  All pointers named "device" must be
+ * device memory of the GPU that was current when the handle was created.  A
+ * `stream` argument is a cudaStream_t passed as void* (NULL = the legacy default
+ * stream).  Every call that takes a stream only enqueues work on it and returns;
+ * the caller synchronizes.  Calls on one handle must not run concurrently.
+ *
+ * Errors.  Functions returning int give 0 on success or a negative code below;
+ * cser_last_error() returns a thread-local message for the last failure.  No call
+ * aborts, throws, or traps on the device.
+ */
+#ifndef CSER_H_
+#define CSER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CSER_OK             0
+#define CSER_ERR_INVALID   -1   /* bad argument (NULL, non-positive size, bad ratio, misuse)   */
+#define CSER_ERR_NOMEM     -2   /* device or host allocation failed                            */
+#define CSER_ERR_CUDA      -3   /* a CUDA runtime call or a kernel launch failed               */
+#define CSER_ERR_TOO_SMALL -4   /* destination / source buffer smaller than the state it holds */
+
+/* `which` of cser_read_state / cser_write_state */
+#define CSER_STATE_X       0    /* fp32 [n, d]  local models                                   */
+#define CSER_STATE_E       1    /* fp32 [n, d]  local errors                                   */
+#define CSER_STATE_M       2    /* fp32 [n, d]  local momenta (only when beta != 0)            */
+#define CSER_STATE_MASK_G  3    /* uint8 [B]    update mask of the last step                   */
+#define CSER_STATE_MASK_R  4    /* uint8 [B]    reset mask of the last reset step              */
+#define CSER_STATE_T       5    /* uint64       step counter t (host value, copied immediately) */
+
+typedef struct cser_ctx *cser_handle;
+
+/*
+ * Create an optimizer state for n_workers x d on the current device (Algorithm 2
+ * line 2 / Algorithm 4 line 2: x = 0 until cser_set_x0, e = 0, m = 0, t = 0).
+ *   d           > 0, elements per worker
+ *   n_workers   > 0
+ *   block_size  > 0, elements per GRBS block (last block may be short)
+ *   R1, R2      >= 1, compression ratios of the update / reset compressors
+ *   H           > 0, error-reset interval
+ *   eta         finite learning rate;  beta in [0, 1): 0 = no momentum (m is not
+ *               allocated, read or written)
+ *   seed        shared GRBS seed
+ * The library owns x, e, m and the masks (about (2 or 3)*n*d*4 bytes of device
+ * memory) until cser_destroy.  Returns NULL on failure.
+ */
+cser_handle cser_create(int64_t d, int32_t n_workers, int32_t block_size,
+                        uint32_t R1, uint32_t R2, int32_t H,
+                        float eta, float beta, uint64_t seed);
+
+/*
+ * Same, for one column slab of a longer vector that several GPUs share by
+ * columns: this handle holds blocks block_begin .. block_begin + ceil(d/block_size) - 1
+ * of the global vector, and draws its masks with those global block ids, so that
+ * every slab sees the mask the whole vector would see (Section 3.3: all workers
+ * pick the same blocks from the synchronized seed).  No data is exchanged.
+ */
+cser_handle cser_create_slab(int64_t d, int32_t n_workers, int32_t block_size,
+                             uint32_t R1, uint32_t R2, int32_t H,
+                             float eta, float beta, uint64_t seed, int64_t block_begin);
+
+/* Free everything the handle owns.  The caller must have synchronized its streams. NULL is ignored. */
+void cser_destroy(cser_handle h);
+
+/*
+ * x_i <- x0 for every worker, e <- 0, m <- 0, t <- 0 (Algorithm 2 line 2).
+ * x0: d fp32 values, host or device memory.
+ */
+int cser_set_x0(cser_handle h, const float *x0, void *stream);
+
+/*
+ * One iteration (Algorithm 2 lines 5-13 / Algorithm 4 lines 5-15) for all workers.
+ * grad: device, fp32 [n, d] row-major with leading dimension d; borrowed, read-only,
+ * must stay valid and unchanged until the work enqueued on `stream` has finished.
+ * Increments t, then enqueues the GRBS mask kernel and the fused step kernel.
+ */
+int cser_step(cser_handle h, const float *grad, void *stream);
+
+/*
+ * The same iteration with the gradients in HOST memory (pinned memory gives
+ * asynchronous copies): the library copies them, slab by slab, into a device
+ * staging buffer it owns (allocated on the first such call, n*d*4 bytes) and runs
+ * the step kernel on each slab as it lands, so copy and compute overlap.
+ * Uses two internal streams that are ordered after `stream` at entry and joined
+ * back into `stream` before returning.
+ */
+int cser_step_host(cser_handle h, const float *grad_host, void *stream);
+
+/*
+ * Copy one piece of state to dst (host or device), enqueued on `stream`.
+ * dst_bytes must be at least the size of the piece: n*d*4 for x/e/m, B for a mask,
+ * 8 for t.  CSER_STATE_M with beta == 0 is CSER_ERR_INVALID.
+ */
+int cser_read_state(cser_handle h, int which, void *dst, size_t dst_bytes, void *stream);
+
+/*
+ * Restore one piece of state from src (host or device) - the inverse of
+ * cser_read_state, for checkpoint/resume.  `bytes` must be exactly the piece's size.
+ * Masks cannot be written (use cser_debug_set_masks).
+ */
+int cser_write_state(cser_handle h, int which, const void *src, size_t bytes, void *stream);
+
+/*
+ * Test hook: the NEXT cser_step uses these block masks (uint8 [B] each, host or
+ * device, non-zero = selected) instead of drawing them.  r_mask may be NULL if
+ * that step is not a reset step.  The copy is enqueued on `stream`.
+ */
+int cser_debug_set_masks(cser_handle h, const uint8_t *g_mask, const uint8_t *r_mask, void *stream);
+
+/*
+ * Stand-alone GRBS block-select kernel (Definition 2): writes uint8 flags of blocks
+ * block_begin .. block_begin + n_blocks - 1 at step t for compressor `which`
+ * (0 = update, 1 = reset) with ratio R into device memory `mask_out`.
+ */
+int cser_grbs_mask(uint64_t seed, uint64_t t, uint32_t which, int64_t block_begin,
+                   int64_t n_blocks, uint32_t R, uint8_t *mask_out, void *stream);
+
+/*
+ * Per-kernel timing.  With on != 0, cser_step brackets its mask kernel and its
+ * fused step kernel with CUDA events on the launching stream.
+ * cser_last_kernel_ms waits for the last step's events and returns both durations
+ * in milliseconds (either pointer may be NULL).
+ */
+int cser_set_timing(cser_handle h, int on);
+int cser_last_kernel_ms(cser_handle h, float *mask_ms, float *step_ms);
+
+/* Number of kernels this library has launched on behalf of the handle. */
+int64_t cser_launch_count(cser_handle h);
+
+/* Thread-local description of the last error in this thread ("" if none). */
+const char *cser_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CSER_H_ */

@@ -1,0 +1,660 @@
+// CSER / M-CSER optimizer step for B200 (sm_100a): GRBS mask kernel, fused step
+// kernel and the C ABI declared in include/cser.h.
+//
+// Layout: g, x, e, m are fp32 [n, d] row-major (worker-major).  A thread owns one
+// vector column (4 consecutive elements, or 1 in the scalar fallback) and walks
+// the worker axis, so every warp access is a contiguous 512-byte run of one row.
+// The step is bound by HBM traffic (about 28 bytes per element and worker against
+// 7 flops), so the kernel is organised around keeping many independent 16-byte
+// loads in flight per thread and touching every byte exactly once; there is no
+// contraction here and tensor cores are not used.
+//
+// Compiled with -fmad=false: every multiply and add rounds separately, in the
+// order stated in include/cser.h.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <stdarg.h>
+#include <string.h>
+#include <math.h>
+#include <new>
+
+#include "cser.h"
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+int fail(int code, const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+#define CU_TRY(expr)                                                                      \
+    do {                                                                                  \
+        cudaError_t _e = (expr);                                                          \
+        if (_e != cudaSuccess)                                                            \
+            return fail(_e == cudaErrorMemoryAllocation ? CSER_ERR_NOMEM : CSER_ERR_CUDA, \
+                        "%s: %s", #expr, cudaGetErrorString(_e));                         \
+    } while (0)
+
+// ------------------------------------------------------------------ Philox4x32-10
+// Salmon et al., SC'11.  Ten rounds; key bumped by the Weyl constants each round.
+__device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t k0, uint32_t k1, uint32_t c0,
+                                                        uint32_t c1, uint32_t c2, uint32_t c3) {
+    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+    const uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+        const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+        c0 = hi1 ^ c1 ^ k0;
+        c1 = lo1;
+        c2 = hi0 ^ c3 ^ k1;
+        c3 = lo0;
+        k0 += W0;
+        k1 += W1;
+    }
+    return c0;
+}
+
+// GRBS block select (Definition 2).  Thread idx < B draws the update mask of block
+// idx, thread B <= idx < 2B the reset mask of block idx - B (only on reset steps).
+__global__ void __launch_bounds__(256)
+grbs_mask_kernel(uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r, long long B,
+                 long long block_begin, uint32_t k0, uint32_t k1, uint32_t t_lo, uint32_t t_hi,
+                 uint32_t R_g, uint32_t R_r, int n_masks, uint32_t first_which) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= B * n_masks) return;
+    const uint32_t second = idx >= B ? 1u : 0u;
+    const long long b = idx - (second ? B : 0);
+    const uint32_t which = first_which + second;
+    const uint32_t R = which ? R_r : R_g;
+    const uint32_t w0 =
+        philox4x32_10_word0(k0, k1, (uint32_t)(block_begin + b), t_lo, t_hi, which);
+    const uint8_t sel = ((unsigned long long)w0 * R < (1ull << 32)) ? 1 : 0;
+    (second ? mask_r : mask_g)[b] = sel;
+}
+
+// ------------------------------------------------------------------ fused step
+template <int V>
+struct Pack {
+    float v[V];
+};
+
+template <int V>
+__device__ __forceinline__ Pack<V> ld(const float *p) {
+    Pack<V> r;
+    if constexpr (V == 4) {
+        const float4 t = *reinterpret_cast<const float4 *>(p);
+        r.v[0] = t.x, r.v[1] = t.y, r.v[2] = t.z, r.v[3] = t.w;
+    } else {
+        r.v[0] = *p;
+    }
+    return r;
+}
+
+// gradients are read exactly once: stream them past the caches
+template <int V>
+__device__ __forceinline__ Pack<V> ld_stream(const float *p) {
+    Pack<V> r;
+    if constexpr (V == 4) {
+        const float4 t = __ldcs(reinterpret_cast<const float4 *>(p));
+        r.v[0] = t.x, r.v[1] = t.y, r.v[2] = t.z, r.v[3] = t.w;
+    } else {
+        r.v[0] = __ldcs(p);
+    }
+    return r;
+}
+
+template <int V>
+__device__ __forceinline__ void st(float *p, const Pack<V> &a) {
+    if constexpr (V == 4) {
+        *reinterpret_cast<float4 *>(p) = make_float4(a.v[0], a.v[1], a.v[2], a.v[3]);
+    } else {
+        *p = a.v[0];
+    }
+}
+
+struct StepParams {
+    const float *g;
+    float *x, *e, *m;
+    const uint8_t *mask_g, *mask_r;
+    long long d;         // elements per row
+    long long c_begin;   // first vector column handled by this launch
+    long long c_end;     // one past the last
+    unsigned bsv;        // GRBS block size in vector columns
+    int n;
+    float eta, beta, n_f;
+};
+
+// Get_p (Appendix A.4) for one pack; updates m in place when MOM.
+template <int V, bool MOM>
+__device__ __forceinline__ Pack<V> get_p(const Pack<V> &g, Pack<V> &m, float eta, float beta) {
+    Pack<V> p;
+#pragma unroll
+    for (int k = 0; k < V; ++k) {
+        if constexpr (MOM) {
+            const float t1 = beta * m.v[k];
+            m.v[k] = t1 + g.v[k];
+            const float t2 = beta * m.v[k];
+            p.v[k] = eta * (t2 + g.v[k]);
+        } else {
+            p.v[k] = eta * g.v[k];
+        }
+    }
+    return p;
+}
+
+// One thread = one vector column, all workers.  U = workers whose loads are
+// issued together before any of their results is used.
+template <int V, bool MOM, bool RESET, int U>
+__global__ void __launch_bounds__(256) cser_step_kernel(const StepParams P) {
+    const long long c = P.c_begin + (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= P.c_end) return;
+    const long long b = (P.c_end <= 0xffffffffll) ? (long long)((uint32_t)c / P.bsv)
+                                                  : (long long)((unsigned long long)c / P.bsv);
+    const bool sg = P.mask_g[b] != 0;
+    const bool sr = RESET ? (P.mask_r[b] != 0) : false;
+    const long long d = P.d;
+    const int n = P.n;
+    const float eta = P.eta, beta = P.beta;
+    const float *__restrict__ g = P.g + c * V;
+    float *__restrict__ x = P.x + c * V;
+    float *__restrict__ e = P.e + c * V;
+    float *__restrict__ m = MOM ? P.m + c * V : nullptr;
+
+    if (!sg && !sr) {
+        // Unselected block, no reset: C(p) = 0, so p' = r = p (Algorithm 3 lines 4-8):
+        // x_i -= p_i, e_i -= p_i.  Purely elementwise.
+        for (int i0 = 0; i0 < n; i0 += U) {
+            Pack<V> gv[U], mv[U], xv[U], ev[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (i0 + u < n) {
+                    const long long o = (long long)(i0 + u) * d;
+                    gv[u] = ld_stream<V>(g + o);
+                    if constexpr (MOM) mv[u] = ld<V>(m + o);
+                    xv[u] = ld<V>(x + o);
+                    ev[u] = ld<V>(e + o);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (i0 + u < n) {
+                    const long long o = (long long)(i0 + u) * d;
+                    const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], eta, beta);
+#pragma unroll
+                    for (int k = 0; k < V; ++k) {
+                        xv[u].v[k] = xv[u].v[k] - p.v[k];
+                        ev[u].v[k] = ev[u].v[k] - p.v[k];
+                    }
+                    if constexpr (MOM) st<V>(m + o, mv[u]);
+                    st<V>(x + o, xv[u]);
+                    st<V>(e + o, ev[u]);
+                }
+            }
+        }
+        return;
+    }
+
+    Pack<V> sum_e;   // sum over workers of e_{t-1/2} (reset-selected columns)
+#pragma unroll
+    for (int k = 0; k < V; ++k) sum_e.v[k] = 0.f;
+
+    if (sg) {
+        // Selected block: r = 0, p' = mean_k p_k.  Pass A forms the mean (and updates m).
+        Pack<V> sum_p;
+#pragma unroll
+        for (int k = 0; k < V; ++k) sum_p.v[k] = 0.f;
+        for (int i = 0; i < n; ++i) {
+            const long long o = (long long)i * d;
+            const Pack<V> gv = ld_stream<V>(g + o);
+            Pack<V> mv;
+            if constexpr (MOM) mv = ld<V>(m + o);
+            const Pack<V> p = get_p<V, MOM>(gv, mv, eta, beta);
+            if constexpr (MOM) st<V>(m + o, mv);
+#pragma unroll
+            for (int k = 0; k < V; ++k) sum_p.v[k] = (i == 0) ? p.v[k] : sum_p.v[k] + p.v[k];
+        }
+        Pack<V> pbar;
+#pragma unroll
+        for (int k = 0; k < V; ++k) pbar.v[k] = sum_p.v[k] / P.n_f;
+        // Pass B: x_i -= p-bar.  On a reset-selected column also fold in x - e and zero e.
+        for (int i = 0; i < n; ++i) {
+            const long long o = (long long)i * d;
+            Pack<V> xv = ld<V>(x + o);
+#pragma unroll
+            for (int k = 0; k < V; ++k) xv.v[k] = xv.v[k] - pbar.v[k];
+            if (sr) {
+                const Pack<V> ev = ld<V>(e + o);
+                Pack<V> z;
+#pragma unroll
+                for (int k = 0; k < V; ++k) {
+                    sum_e.v[k] = (i == 0) ? ev.v[k] : sum_e.v[k] + ev.v[k];
+                    xv.v[k] = xv.v[k] - ev.v[k];
+                    z.v[k] = 0.f;
+                }
+                st<V>(e + o, z);
+            }
+            st<V>(x + o, xv);
+        }
+    } else {
+        // Unselected by the update mask but reset-selected: x_{t-1/2} = x - p,
+        // e_{t-1/2} = e - p; store x_{t-1/2} - e_{t-1/2}, accumulate e_{t-1/2}, zero e.
+        for (int i = 0; i < n; ++i) {
+            const long long o = (long long)i * d;
+            const Pack<V> gv = ld_stream<V>(g + o);
+            Pack<V> mv;
+            if constexpr (MOM) mv = ld<V>(m + o);
+            Pack<V> xv = ld<V>(x + o);
+            const Pack<V> ev = ld<V>(e + o);
+            const Pack<V> p = get_p<V, MOM>(gv, mv, eta, beta);
+            if constexpr (MOM) st<V>(m + o, mv);
+            Pack<V> z;
+#pragma unroll
+            for (int k = 0; k < V; ++k) {
+                const float xh = xv.v[k] - p.v[k];
+                const float eh = ev.v[k] - p.v[k];
+                sum_e.v[k] = (i == 0) ? eh : sum_e.v[k] + eh;
+                xv.v[k] = xh - eh;
+                z.v[k] = 0.f;
+            }
+            st<V>(x + o, xv);
+            st<V>(e + o, z);
+        }
+    }
+
+    if (sr) {
+        // Error reset (Algorithm 2 lines 11-12): x_i = (x_{t-1/2} - e_{t-1/2}) + mean_k e_k.
+        Pack<V> ebar;
+#pragma unroll
+        for (int k = 0; k < V; ++k) ebar.v[k] = sum_e.v[k] / P.n_f;
+        for (int i = 0; i < n; ++i) {
+            const long long o = (long long)i * d;
+            Pack<V> xv = ld<V>(x + o);
+#pragma unroll
+            for (int k = 0; k < V; ++k) xv.v[k] = xv.v[k] + ebar.v[k];
+            st<V>(x + o, xv);
+        }
+    }
+}
+
+// x_i <- x0 for all workers; e, m <- 0
+__global__ void __launch_bounds__(256)
+broadcast_x0_kernel(const float *__restrict__ x0, float *__restrict__ x, float *__restrict__ e,
+                    float *__restrict__ m, long long d, int n) {
+    const long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= d) return;
+    const float v = x0[j];
+    for (int i = 0; i < n; ++i) {
+        const long long o = (long long)i * d + j;
+        x[o] = v;
+        e[o] = 0.f;
+        if (m) m[o] = 0.f;
+    }
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ handle
+struct cser_ctx {
+    long long d = 0, B = 0, block_begin = 0;
+    int n = 0, bs = 0, H = 0, device = 0;
+    uint32_t R1 = 1, R2 = 1;
+    float eta = 0.f, beta = 0.f;
+    uint64_t seed = 0, t = 0;
+    float *x = nullptr, *e = nullptr, *m = nullptr;
+    uint8_t *mask_g = nullptr, *mask_r = nullptr;
+    float *x0_stage = nullptr;                       // [d] staging for a host x0
+    bool masks_injected = false;
+    bool vec4 = false;                               // 128-bit path usable for the state arrays
+    // timing
+    bool timing = false;
+    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+    bool ev_valid = false;
+    long long launches = 0;
+    // host-gradient path
+    float *g_stage = nullptr;
+    cudaStream_t hs[2] = {nullptr, nullptr};
+    cudaEvent_t h_ev[4] = {nullptr, nullptr, nullptr, nullptr};
+};
+
+namespace {
+
+size_t state_elems(const cser_ctx *h) { return (size_t)h->n * (size_t)h->d; }
+
+int launch_masks(cser_ctx *h, bool is_reset, cudaStream_t s) {
+    const int n_masks = is_reset ? 2 : 1;
+    const long long total = h->B * n_masks;
+    const unsigned grid = (unsigned)((total + 255) / 256);
+    grbs_mask_kernel<<<grid, 256, 0, s>>>(h->mask_g, h->mask_r, h->B, h->block_begin,
+                                          (uint32_t)(h->seed & 0xffffffffu), (uint32_t)(h->seed >> 32),
+                                          (uint32_t)(h->t & 0xffffffffu), (uint32_t)(h->t >> 32),
+                                          h->R1, h->R2, n_masks, 0u);
+    h->launches++;
+    CU_TRY(cudaGetLastError());
+    return CSER_OK;
+}
+
+template <int V, int U>
+int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t s) {
+    const long long cols = P.c_end - P.c_begin;
+    if (cols <= 0) return CSER_OK;
+    const long long grid_ll = (cols + 255) / 256;
+    if (grid_ll > 0x7fffffffll) return fail(CSER_ERR_INVALID, "vector too long for one launch");
+    const unsigned grid = (unsigned)grid_ll;
+    const bool mom = h->m != nullptr;
+    if (mom) {
+        if (is_reset) cser_step_kernel<V, true, true, U><<<grid, 256, 0, s>>>(P);
+        else          cser_step_kernel<V, true, false, U><<<grid, 256, 0, s>>>(P);
+    } else {
+        if (is_reset) cser_step_kernel<V, false, true, U><<<grid, 256, 0, s>>>(P);
+        else          cser_step_kernel<V, false, false, U><<<grid, 256, 0, s>>>(P);
+    }
+    h->launches++;
+    CU_TRY(cudaGetLastError());
+    return CSER_OK;
+}
+
+// Launch the fused step kernel on element columns [col0, col1) of gradients `grad`.
+int launch_step(cser_ctx *h, const float *grad, long long col0, long long col1, bool is_reset,
+                cudaStream_t s) {
+    StepParams P;
+    P.g = grad, P.x = h->x, P.e = h->e, P.m = h->m;
+    P.mask_g = h->mask_g, P.mask_r = h->mask_r;
+    P.d = h->d, P.n = h->n;
+    P.eta = h->eta, P.beta = h->beta, P.n_f = (float)h->n;
+    const bool v4 = h->vec4 && ((uintptr_t)grad % 16 == 0) && (col0 % 4 == 0) &&
+                    (col1 % 4 == 0 || col1 == h->d);
+    if (v4) {
+        P.c_begin = col0 / 4, P.c_end = col1 / 4, P.bsv = (unsigned)(h->bs / 4);
+        return launch_step_v<4, 2>(h, P, is_reset, s);
+    }
+    P.c_begin = col0, P.c_end = col1, P.bsv = (unsigned)h->bs;
+    return launch_step_v<1, 4>(h, P, is_reset, s);
+}
+
+int check_handle(cser_ctx *h) {
+    if (!h) return fail(CSER_ERR_INVALID, "NULL handle");
+    int dev = -1;
+    CU_TRY(cudaGetDevice(&dev));
+    if (dev != h->device)
+        return fail(CSER_ERR_INVALID, "handle belongs to device %d, current device is %d", h->device, dev);
+    return CSER_OK;
+}
+
+int check_device_ptr(const void *p, const char *what) {
+    if (!p) return fail(CSER_ERR_INVALID, "%s is NULL", what);
+    cudaPointerAttributes a;
+    cudaError_t er = cudaPointerGetAttributes(&a, p);
+    if (er != cudaSuccess) {
+        cudaGetLastError();
+        return fail(CSER_ERR_INVALID, "%s: cannot query pointer (%s)", what, cudaGetErrorString(er));
+    }
+    if (a.type != cudaMemoryTypeDevice && a.type != cudaMemoryTypeManaged)
+        return fail(CSER_ERR_INVALID, "%s must be device memory", what);
+    return CSER_OK;
+}
+
+// advance t and decide whether this iteration resets (Algorithm 2 line 8)
+bool begin_iteration(cser_ctx *h) {
+    h->t += 1;
+    return (h->t % (uint64_t)h->H) == 0;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ C ABI
+extern "C" {
+
+const char *cser_last_error(void) { return g_err; }
+
+cser_handle cser_create_slab(int64_t d, int32_t n_workers, int32_t block_size, uint32_t R1,
+                             uint32_t R2, int32_t H, float eta, float beta, uint64_t seed,
+                             int64_t block_begin) {
+    g_err[0] = 0;
+    if (d <= 0 || n_workers <= 0 || block_size <= 0 || R1 == 0 || R2 == 0 || H <= 0 ||
+        block_begin < 0) {
+        fail(CSER_ERR_INVALID, "cser_create: d, n_workers, block_size, R1, R2, H must be positive");
+        return nullptr;
+    }
+    if (!isfinite(eta) || !(beta >= 0.f && beta < 1.f)) {
+        fail(CSER_ERR_INVALID, "cser_create: eta must be finite and beta in [0, 1)");
+        return nullptr;
+    }
+    const long long B = (d + block_size - 1) / block_size;
+    if (block_begin + B > 0xffffffffll) {
+        fail(CSER_ERR_INVALID, "cser_create: more than 2^32 blocks");
+        return nullptr;
+    }
+    cser_ctx *h = new (std::nothrow) cser_ctx();
+    if (!h) {
+        fail(CSER_ERR_NOMEM, "cser_create: host allocation failed");
+        return nullptr;
+    }
+    h->d = d, h->n = n_workers, h->bs = block_size, h->R1 = R1, h->R2 = R2, h->H = H;
+    h->eta = eta, h->beta = beta, h->seed = seed, h->B = B, h->block_begin = block_begin;
+    h->vec4 = (d % 4 == 0) && (block_size % 4 == 0);
+    const size_t bytes = state_elems(h) * sizeof(float);
+    cudaError_t er = cudaGetDevice(&h->device);
+    if (er == cudaSuccess) er = cudaMalloc(&h->x, bytes);
+    if (er == cudaSuccess) er = cudaMalloc(&h->e, bytes);
+    if (er == cudaSuccess && beta != 0.f) er = cudaMalloc(&h->m, bytes);
+    if (er == cudaSuccess) er = cudaMalloc(&h->mask_g, (size_t)B);
+    if (er == cudaSuccess) er = cudaMalloc(&h->mask_r, (size_t)B);
+    if (er == cudaSuccess) er = cudaMemset(h->x, 0, bytes);
+    if (er == cudaSuccess) er = cudaMemset(h->e, 0, bytes);
+    if (er == cudaSuccess && h->m) er = cudaMemset(h->m, 0, bytes);
+    if (er == cudaSuccess) er = cudaMemset(h->mask_g, 0, (size_t)B);
+    if (er == cudaSuccess) er = cudaMemset(h->mask_r, 0, (size_t)B);
+    for (int k = 0; k < 3 && er == cudaSuccess; ++k) er = cudaEventCreate(&h->ev[k]);
+    if (er == cudaSuccess) er = cudaDeviceSynchronize();
+    if (er != cudaSuccess) {
+        fail(er == cudaErrorMemoryAllocation ? CSER_ERR_NOMEM : CSER_ERR_CUDA, "cser_create: %s",
+             cudaGetErrorString(er));
+        cudaGetLastError();
+        cser_destroy(h);
+        return nullptr;
+    }
+    return h;
+}
+
+cser_handle cser_create(int64_t d, int32_t n_workers, int32_t block_size, uint32_t R1, uint32_t R2,
+                        int32_t H, float eta, float beta, uint64_t seed) {
+    return cser_create_slab(d, n_workers, block_size, R1, R2, H, eta, beta, seed, 0);
+}
+
+void cser_destroy(cser_handle h) {
+    if (!h) return;
+    cudaFree(h->x), cudaFree(h->e), cudaFree(h->m);
+    cudaFree(h->mask_g), cudaFree(h->mask_r), cudaFree(h->x0_stage), cudaFree(h->g_stage);
+    for (auto &ev : h->ev) if (ev) cudaEventDestroy(ev);
+    for (auto &ev : h->h_ev) if (ev) cudaEventDestroy(ev);
+    for (auto &s : h->hs) if (s) cudaStreamDestroy(s);
+    delete h;
+}
+
+int cser_set_x0(cser_handle h, const float *x0, void *stream) {
+    if (int rc = check_handle(h)) return rc;
+    if (!x0) return fail(CSER_ERR_INVALID, "cser_set_x0: x0 is NULL");
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaPointerAttributes a;
+    cudaError_t er = cudaPointerGetAttributes(&a, x0);
+    if (er != cudaSuccess) cudaGetLastError();
+    const float *src = x0;
+    if (er != cudaSuccess || (a.type != cudaMemoryTypeDevice && a.type != cudaMemoryTypeManaged)) {
+        if (!h->x0_stage) CU_TRY(cudaMalloc(&h->x0_stage, (size_t)h->d * sizeof(float)));
+        CU_TRY(cudaMemcpyAsync(h->x0_stage, x0, (size_t)h->d * sizeof(float), cudaMemcpyHostToDevice, s));
+        src = h->x0_stage;
+    }
+    const unsigned grid = (unsigned)((h->d + 255) / 256);
+    broadcast_x0_kernel<<<grid, 256, 0, s>>>(src, h->x, h->e, h->m, h->d, h->n);
+    h->launches++;
+    CU_TRY(cudaGetLastError());
+    h->t = 0;
+    h->masks_injected = false;
+    return CSER_OK;
+}
+
+int cser_step(cser_handle h, const float *grad, void *stream) {
+    if (int rc = check_handle(h)) return rc;
+    if (int rc = check_device_ptr(grad, "cser_step: grad")) return rc;
+    if ((uintptr_t)grad % 4 != 0) return fail(CSER_ERR_INVALID, "cser_step: grad is not 4-byte aligned");
+    cudaStream_t s = (cudaStream_t)stream;
+    const bool is_reset = begin_iteration(h);
+    if (h->timing) CU_TRY(cudaEventRecord(h->ev[0], s));
+    if (!h->masks_injected) {
+        if (int rc = launch_masks(h, is_reset, s)) return rc;
+    }
+    h->masks_injected = false;
+    if (h->timing) CU_TRY(cudaEventRecord(h->ev[1], s));
+    if (int rc = launch_step(h, grad, 0, h->d, is_reset, s)) return rc;
+    if (h->timing) {
+        CU_TRY(cudaEventRecord(h->ev[2], s));
+        h->ev_valid = true;
+    }
+    return CSER_OK;
+}
+
+int cser_step_host(cser_handle h, const float *grad_host, void *stream) {
+    if (int rc = check_handle(h)) return rc;
+    if (!grad_host) return fail(CSER_ERR_INVALID, "cser_step_host: grad_host is NULL");
+    cudaStream_t s = (cudaStream_t)stream;
+    if (!h->g_stage) {
+        CU_TRY(cudaMalloc(&h->g_stage, state_elems(h) * sizeof(float)));
+        for (auto &st_ : h->hs) CU_TRY(cudaStreamCreateWithFlags(&st_, cudaStreamNonBlocking));
+        for (auto &ev : h->h_ev) CU_TRY(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+    }
+    const bool is_reset = begin_iteration(h);
+    // masks first, on the caller's stream; both internal streams start after them
+    if (!h->masks_injected) {
+        if (int rc = launch_masks(h, is_reset, s)) return rc;
+    }
+    h->masks_injected = false;
+    CU_TRY(cudaEventRecord(h->h_ev[0], s));
+    CU_TRY(cudaStreamWaitEvent(h->hs[0], h->h_ev[0], 0));
+    CU_TRY(cudaStreamWaitEvent(h->hs[1], h->h_ev[0], 0));
+    // column slabs of about 64 MB of gradients each, boundaries on multiples of 1024 columns
+    const long long d = h->d;
+    long long n_slabs = (long long)((state_elems(h) * sizeof(float) + (64u << 20) - 1) / (64u << 20));
+    if (n_slabs < 1) n_slabs = 1;
+    if (n_slabs > 256) n_slabs = 256;
+    long long slab = ((d + n_slabs - 1) / n_slabs + 1023) / 1024 * 1024;
+    int k = 0;
+    for (long long c0 = 0; c0 < d; c0 += slab, ++k) {
+        const long long c1 = (c0 + slab < d) ? c0 + slab : d;
+        cudaStream_t cs = h->hs[k & 1];
+        CU_TRY(cudaMemcpy2DAsync(h->g_stage + c0, (size_t)d * sizeof(float), grad_host + c0,
+                                 (size_t)d * sizeof(float), (size_t)(c1 - c0) * sizeof(float),
+                                 (size_t)h->n, cudaMemcpyHostToDevice, cs));
+        if (int rc = launch_step(h, h->g_stage, c0, c1, is_reset, cs)) return rc;
+    }
+    CU_TRY(cudaEventRecord(h->h_ev[1], h->hs[0]));
+    CU_TRY(cudaEventRecord(h->h_ev[2], h->hs[1]));
+    CU_TRY(cudaStreamWaitEvent(s, h->h_ev[1], 0));
+    CU_TRY(cudaStreamWaitEvent(s, h->h_ev[2], 0));
+    return CSER_OK;
+}
+
+static int state_piece(cser_ctx *h, int which, void **ptr, size_t *bytes) {
+    switch (which) {
+        case CSER_STATE_X: *ptr = h->x, *bytes = state_elems(h) * sizeof(float); return CSER_OK;
+        case CSER_STATE_E: *ptr = h->e, *bytes = state_elems(h) * sizeof(float); return CSER_OK;
+        case CSER_STATE_M:
+            if (!h->m) return fail(CSER_ERR_INVALID, "no momentum state (beta == 0)");
+            *ptr = h->m, *bytes = state_elems(h) * sizeof(float);
+            return CSER_OK;
+        case CSER_STATE_MASK_G: *ptr = h->mask_g, *bytes = (size_t)h->B; return CSER_OK;
+        case CSER_STATE_MASK_R: *ptr = h->mask_r, *bytes = (size_t)h->B; return CSER_OK;
+        case CSER_STATE_T: *ptr = nullptr, *bytes = sizeof(uint64_t); return CSER_OK;
+        default: return fail(CSER_ERR_INVALID, "unknown state id %d", which);
+    }
+}
+
+int cser_read_state(cser_handle h, int which, void *dst, size_t dst_bytes, void *stream) {
+    if (int rc = check_handle(h)) return rc;
+    if (!dst) return fail(CSER_ERR_INVALID, "cser_read_state: dst is NULL");
+    void *src;
+    size_t bytes;
+    if (int rc = state_piece(h, which, &src, &bytes)) return rc;
+    if (dst_bytes < bytes)
+        return fail(CSER_ERR_TOO_SMALL, "cser_read_state: need %zu bytes, got %zu", bytes, dst_bytes);
+    if (which == CSER_STATE_T) {
+        CU_TRY(cudaMemcpy(dst, &h->t, sizeof(uint64_t), cudaMemcpyDefault));
+        return CSER_OK;
+    }
+    CU_TRY(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, (cudaStream_t)stream));
+    return CSER_OK;
+}
+
+int cser_write_state(cser_handle h, int which, const void *src, size_t bytes, void *stream) {
+    if (int rc = check_handle(h)) return rc;
+    if (!src) return fail(CSER_ERR_INVALID, "cser_write_state: src is NULL");
+    if (which == CSER_STATE_MASK_G || which == CSER_STATE_MASK_R)
+        return fail(CSER_ERR_INVALID, "masks cannot be written; use cser_debug_set_masks");
+    void *dst;
+    size_t want;
+    if (int rc = state_piece(h, which, &dst, &want)) return rc;
+    if (bytes != want)
+        return fail(CSER_ERR_TOO_SMALL, "cser_write_state: need exactly %zu bytes, got %zu", want, bytes);
+    if (which == CSER_STATE_T) {
+        CU_TRY(cudaMemcpy(&h->t, src, sizeof(uint64_t), cudaMemcpyDefault));
+        return CSER_OK;
+    }
+    CU_TRY(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, (cudaStream_t)stream));
+    return CSER_OK;
+}
+
+int cser_debug_set_masks(cser_handle h, const uint8_t *g_mask, const uint8_t *r_mask, void *stream) {
+    if (int rc = check_handle(h)) return rc;
+    if (!g_mask) return fail(CSER_ERR_INVALID, "cser_debug_set_masks: g_mask is NULL");
+    const bool next_is_reset = ((h->t + 1) % (uint64_t)h->H) == 0;
+    if (next_is_reset && !r_mask)
+        return fail(CSER_ERR_INVALID, "cser_debug_set_masks: next step resets, r_mask is NULL");
+    cudaStream_t s = (cudaStream_t)stream;
+    CU_TRY(cudaMemcpyAsync(h->mask_g, g_mask, (size_t)h->B, cudaMemcpyDefault, s));
+    if (r_mask) CU_TRY(cudaMemcpyAsync(h->mask_r, r_mask, (size_t)h->B, cudaMemcpyDefault, s));
+    h->masks_injected = true;
+    return CSER_OK;
+}
+
+int cser_grbs_mask(uint64_t seed, uint64_t t, uint32_t which, int64_t block_begin, int64_t n_blocks,
+                   uint32_t R, uint8_t *mask_out, void *stream) {
+    if (n_blocks < 0 || block_begin < 0 || R == 0 || which > 1 || block_begin + n_blocks > 0xffffffffll)
+        return fail(CSER_ERR_INVALID, "cser_grbs_mask: bad arguments");
+    if (n_blocks == 0) return CSER_OK;
+    if (int rc = check_device_ptr(mask_out, "cser_grbs_mask: mask_out")) return rc;
+    const unsigned grid = (unsigned)((n_blocks + 255) / 256);
+    grbs_mask_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(
+        mask_out, mask_out, n_blocks, block_begin, (uint32_t)(seed & 0xffffffffu),
+        (uint32_t)(seed >> 32), (uint32_t)(t & 0xffffffffu), (uint32_t)(t >> 32), R, R, 1, which);
+    CU_TRY(cudaGetLastError());
+    return CSER_OK;
+}
+
+int cser_set_timing(cser_handle h, int on) {
+    if (int rc = check_handle(h)) return rc;
+    h->timing = on != 0;
+    h->ev_valid = false;
+    return CSER_OK;
+}
+
+int cser_last_kernel_ms(cser_handle h, float *mask_ms, float *step_ms) {
+    if (int rc = check_handle(h)) return rc;
+    if (!h->ev_valid) return fail(CSER_ERR_INVALID, "no timed step recorded");
+    CU_TRY(cudaEventSynchronize(h->ev[2]));
+    float a = 0.f, b = 0.f;
+    CU_TRY(cudaEventElapsedTime(&a, h->ev[0], h->ev[1]));
+    CU_TRY(cudaEventElapsedTime(&b, h->ev[1], h->ev[2]));
+    if (mask_ms) *mask_ms = a;
+    if (step_ms) *step_ms = b;
+    return CSER_OK;
+}
+
+int64_t cser_launch_count(cser_handle h) { return h ? h->launches : 0; }
+
+}  // extern "C"

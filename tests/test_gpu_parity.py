@@ -1,0 +1,389 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle.
+
+Bars: GRBS masks bit-exact; float state within 1e-6 relative + 1e-7 absolute after
+one step and 1e-4 relative (+ 1e-4 * RMS absolute, for entries that pass near zero)
+after the full run, against the float64 oracle.  Because the kernel is compiled
+without fused multiply-add and follows the same operation order, it must in addition
+equal the float32 evaluation of the oracle exactly (signed zeros compare equal).
+"""
+import ctypes
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from _golden import read_hand_example
+from oracle import CSEROracle, grbs_mask, n_blocks, philox4x32_10, STREAM_GRAD, STREAM_RESET
+from paper_2007_13221_b200 import binding as b, synth
+
+pytestmark = pytest.mark.gpu
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    import __graft_entry__
+    __graft_entry__.build()
+    torch.cuda.set_device(0)
+
+
+def _within(got, want, rtol, atol):
+    return np.abs(got.astype(np.float64) - want) <= rtol * np.abs(want) + atol
+
+
+# ------------------------------------------------------------------ masks
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+def test_mask_kernel_bit_exact_all_configs(cfg):
+    w = synth.CONFIGS[cfg]
+    B = w.n_blocks
+    out = torch.empty(B, dtype=torch.uint8, device=DEV)
+    for seed in (0, 0xDEADBEEF12345678):
+        for t in (1, 2, w.H, 99, 2**32 + 5):
+            for which, R in ((STREAM_GRAD, w.R1), (STREAM_RESET, w.R2)):
+                b.cser_grbs_mask(seed, t, which, 0, B, R, out)
+                assert np.array_equal(out.cpu().numpy(), grbs_mask(seed, t, which, B, R)), (seed, t, which)
+    # slab with global block ids
+    b.cser_grbs_mask(3, 7, 0, 1000, min(B, 3000) - 1000, w.R1, out)
+    assert np.array_equal(out[: min(B, 3000) - 1000].cpu().numpy(),
+                          grbs_mask(3, 7, 0, min(B, 3000) - 1000, w.R1, block_begin=1000))
+
+
+def test_mask_kernel_odd_ratios_and_R1():
+    out = torch.empty(5001, dtype=torch.uint8, device=DEV)
+    for R in (1, 3, 7, 1000, 2**31 + 1, 2**32 - 1):
+        b.cser_grbs_mask(9, 4, 1, 0, 5001, R, out)
+        assert np.array_equal(out.cpu().numpy(), grbs_mask(9, 4, 1, 5001, R))
+
+
+def test_oracle_philox_matches_curand_library():
+    """cuRAND's Philox4_32_10: key = seed, counter = (offset/4 as 64 bits, subsequence as 64 bits)."""
+    L = ctypes.CDLL(os.path.join(ROOT, "tests", "libcurand_philox_check.so"))
+    L.curand_philox_words.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int, ctypes.c_void_p]
+    rng = np.random.default_rng(0)
+    n = 4096
+    seed = rng.integers(0, 2**63, n, dtype=np.int64)
+    subseq = rng.integers(0, 2**63, n, dtype=np.int64)
+    blockctr = rng.integers(0, 2**61, n, dtype=np.int64)
+    seed[0] = subseq[0] = blockctr[0] = 0
+    ts, tq, to = (torch.from_numpy(a).to(DEV) for a in (seed, subseq, blockctr * 4))
+    out = torch.zeros(4 * n, dtype=torch.int32, device=DEV)
+    rc = L.curand_philox_words(ts.data_ptr(), tq.data_ptr(), to.data_ptr(), out.data_ptr(), n, None)
+    torch.cuda.synchronize()
+    assert rc == 0
+    got = out.cpu().numpy().view(np.uint32).reshape(n, 4)
+    u = lambda a: a.astype(np.uint64)
+    want = philox4x32_10(u(seed) & 0xFFFFFFFF, u(seed) >> 32, u(blockctr) & 0xFFFFFFFF, u(blockctr) >> 32,
+                         u(subseq) & 0xFFFFFFFF, u(subseq) >> 32)
+    assert np.array_equal(got, np.stack(want, 1))
+
+
+# ------------------------------------------------------------------ small shapes, element by element
+def _run_both(d, n, bs, R1, R2, H, eta, beta, steps, seed=3, masks=None, x0=None, grads=None, dtype=np.float32):
+    rng = np.random.default_rng(1000 + d + n)
+    x0 = rng.standard_normal(d).astype(np.float32) if x0 is None else x0
+    opt = b.CSER(d, n, bs, R1, R2, H, eta, beta, seed)
+    ref = CSEROracle(d, n, bs, R1, R2, H, eta, beta, seed, dtype=dtype)
+    opt.set_x0(torch.from_numpy(x0).to(DEV))
+    ref.set_x0(x0)
+    for t in range(1, steps + 1):
+        g = (rng.standard_normal(d)[None, :] + 0.5 * rng.standard_normal((n, d))).astype(np.float32) \
+            if grads is None else grads[t - 1]
+        if masks is not None:
+            mg, mr = masks[t - 1]
+            opt.inject_masks(torch.tensor(mg, dtype=torch.uint8, device=DEV),
+                             None if mr is None else torch.tensor(mr, dtype=torch.uint8, device=DEV))
+            ref.inject_masks(mg, mr)
+        opt.step(torch.from_numpy(g).to(DEV))
+        ref.step(g)
+        assert np.array_equal(opt.state(b.STATE_MASK_G).cpu().numpy(), ref.mask_g)
+        if t % H == 0:
+            assert np.array_equal(opt.state(b.STATE_MASK_R).cpu().numpy(), ref.mask_r)
+    return opt, ref
+
+
+SHAPES = [
+    # d, n, bs, R1, R2, H, beta
+    (4096 + 40, 8, 256, 4, 4, 4, 0.0),        # vector path, ragged last block
+    (4096 + 40, 8, 256, 4, 2, 3, 0.9),
+    (20_000, 16, 1024, 2, 2, 2, 0.9),         # several CTAs, n = 16
+    (1001, 3, 7, 2, 2, 2, 0.9),               # scalar path: d and bs not multiples of 4
+    (999, 2, 1000, 2, 2, 1, 0.0),             # B = 1, H = 1
+    (130, 1, 4, 3, 5, 2, 0.9),                # single worker, odd ratios
+    (2048, 5, 4, 1, 1, 3, 0.9),               # R = 1: everything selected, smallest vector block
+    (8, 8, 4, 2, 2, 1, 0.5),                  # tiny
+    (262_144 + 4, 8, 512, 32, 32, 8, 0.9),    # many tiles, tail of one vector column
+]
+
+
+@pytest.mark.parametrize("d,n,bs,R1,R2,H,beta", SHAPES)
+def test_small_shapes_equal_float32_oracle_exactly(d, n, bs, R1, R2, H, beta):
+    opt, ref = _run_both(d, n, bs, R1, R2, H, 0.1, beta, steps=13)
+    for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e")) + (((b.STATE_M, "m"),) if beta else ()):
+        got = opt.state(which).cpu().numpy()
+        want = getattr(ref, name)
+        assert got.shape == want.shape
+        bad = got != want
+        assert not bad.any(), (name, int(bad.sum()), np.argwhere(bad)[:5])
+    assert opt.t == 13
+    opt.close()
+
+
+@pytest.mark.parametrize("d,n,bs,R1,R2,H,beta", SHAPES[:4])
+def test_small_shapes_within_stated_tolerance_of_float64_oracle(d, n, bs, R1, R2, H, beta):
+    for steps, rtol, atol_rms in ((1, 1e-6, None), (100, 1e-4, 1e-4)):
+        opt, ref = _run_both(d, n, bs, R1, R2, H, 0.1, beta, steps=steps, dtype=np.float64)
+        for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e")) + (((b.STATE_M, "m"),) if beta else ()):
+            got = opt.state(which).cpu().numpy()
+            want = getattr(ref, name)
+            atol = 1e-7 if atol_rms is None else atol_rms * float(np.sqrt((want**2).mean()))
+            assert _within(got, want, rtol, atol).all(), (steps, name)
+        opt.close()
+
+
+@pytest.mark.parametrize("beta", [0.0, 0.5])
+def test_hand_worked_example_on_gpu(beta):
+    gold = read_hand_example()
+    g = [np.array([[1, 2, -1, 0], [3, -2, 1, 4]], np.float32), np.array([[2, 2, 2, 2], [0, 4, -2, 6]], np.float32)]
+    masks = [([1, 0], None), ([0, 1], [0, 1])]
+    opt = b.CSER(4, 2, 2, 7, 7, 2, 0.5, beta, 0)
+    opt.set_x0(torch.tensor([1, 2, 3, 4], dtype=torch.float32, device=DEV))
+    for t in (1, 2):
+        mg, mr = masks[t - 1]
+        opt.inject_masks(torch.tensor(mg, dtype=torch.uint8, device=DEV),
+                         None if mr is None else torch.tensor(mr, dtype=torch.uint8, device=DEV))
+        opt.step(torch.from_numpy(g[t - 1]).to(DEV))
+        for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e")) + (((b.STATE_M, "m"),) if beta else ()):
+            got = opt.state(which).cpu().numpy()
+            for i in range(2):
+                assert np.array_equal(got[i], np.array(gold[(beta, t, name, i)], np.float32)), (t, name, i)
+    opt.close()
+
+
+def test_all_four_mask_combinations_on_one_reset_step():
+    """Blocks in neither / update only / reset only / both masks, vector and scalar paths."""
+    for d, bs in ((64, 16), (62, 15)):
+        B = n_blocks(d, bs)
+        mg = [0, 1, 0, 1, 1][:B]
+        mr = [0, 0, 1, 1, 0][:B]
+        masks = [(mg, mr)] * 3
+        opt, ref = _run_both(d, 4, bs, 2, 2, 1, 0.1, 0.9, steps=3, masks=masks)
+        for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e"), (b.STATE_M, "m")):
+            assert np.array_equal(opt.state(which).cpu().numpy(), getattr(ref, name)), (d, name)
+        opt.close()
+
+
+# ------------------------------------------------------------------ full-size workloads
+def _sample_blocks(w, ref_masks_g, ref_masks_r, rng, n_random):
+    B = w.n_blocks
+    blocks = {0, B - 1, B // 2}
+    # blocks whose elements straddle a 2^31-element boundary of the flattened [n, d] index
+    flat = 2**31
+    while flat < w.n_workers * w.d:
+        col = flat % w.d
+        blocks.update({col // w.block_size, max(col // w.block_size - 1, 0)})
+        flat += 2**31
+    blocks.update(int(v) for v in rng.integers(0, B, n_random))
+    for masks in (ref_masks_g, ref_masks_r):
+        for m in masks:
+            sel = np.flatnonzero(m)
+            if sel.size:
+                blocks.update(int(v) for v in rng.choice(sel, min(8, sel.size), replace=False))
+    return np.array(sorted(blocks), dtype=np.int64)
+
+
+def _cols_of(blocks, w):
+    parts = [np.arange(bk * w.block_size, min((bk + 1) * w.block_size, w.d), dtype=np.int64) for bk in blocks]
+    return np.concatenate(parts)
+
+
+def _full_size_parity(cfg, steps=None, n_random=192):
+    w = synth.CONFIGS[cfg]
+    steps = w.steps if steps is None else steps
+    rng = np.random.default_rng(cfg)
+    B = w.n_blocks
+    masks_g = [grbs_mask(w.seed, t, STREAM_GRAD, B, w.R1) for t in range(1, steps + 1)]
+    masks_r = [grbs_mask(w.seed, t, STREAM_RESET, B, w.R2) for t in range(1, steps + 1) if t % w.H == 0]
+    blocks = _sample_blocks(w, masks_g[::max(1, steps // 8)], masks_r[::max(1, len(masks_r) // 8)], rng, n_random)
+    cols = _cols_of(blocks, w)
+    cols_dev = torch.from_numpy(cols).to(DEV)
+    refs = {dt: CSEROracle(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
+                           dtype=dt, cols=cols) for dt in (np.float32, np.float64)}
+    opt = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed)
+    x0 = synth.x0(w, DEV)
+    opt.set_x0(x0)
+    x0_s = x0[cols_dev].cpu().numpy()
+    for r in refs.values():
+        r.set_x0(x0_s)
+    g = torch.empty((w.n_workers, w.d), dtype=torch.float32, device=DEV)
+    buf = torch.empty((w.n_workers, w.d), dtype=torch.float32, device=DEV)
+    names = ((b.STATE_X, "x"), (b.STATE_E, "e")) + (((b.STATE_M, "m"),) if w.beta else ())
+
+    def compare(rtol, atol_abs, atol_rms):
+        for which, name in names:
+            b.cser_read_state(opt.h, which, buf)
+            got = buf[:, cols_dev].cpu().numpy()
+            want32, want64 = refs[np.float32].__dict__[name], refs[np.float64].__dict__[name]
+            atol = atol_abs + atol_rms * float(np.sqrt((want64**2).mean()))
+            assert _within(got, want64, rtol, atol).all(), (cfg, name, "float64 tolerance")
+            bad = got != want32
+            assert not bad.any(), (cfg, name, "float32 exact", int(bad.sum()))
+
+    for t in range(1, steps + 1):
+        synth.gradients(w, t, DEV, out=g)
+        opt.step(g)
+        g_s = g[:, cols_dev].cpu().numpy()
+        for r in refs.values():
+            r.step(g_s)
+        if t == 1:
+            compare(1e-6, 1e-7, 0.0)
+        if t in (1, w.H, steps):
+            assert np.array_equal(opt.state(b.STATE_MASK_G).cpu().numpy(), masks_g[t - 1]), t
+    compare(1e-4, 0.0, 1e-4)
+    # properties that hold at any size, on the whole state: Lemma 1 and zero error after reset
+    b.cser_read_state(opt.h, b.STATE_X, buf)
+    b.cser_read_state(opt.h, b.STATE_E, g)
+    diff = buf - g
+    spread = (diff - diff[0:1]).abs().max().item()
+    assert spread <= 1e-4 * max(1.0, buf.abs().max().item()), spread
+    if steps % w.H == 0:
+        mr = torch.from_numpy(masks_r[-1]).to(DEV).bool()
+        sel_cols = mr.repeat_interleave(w.block_size)[: w.d]
+        assert g[:, sel_cols].abs().max().item() == 0.0
+    assert opt.t == steps
+    opt.close()
+    del g, buf
+    torch.cuda.empty_cache()
+
+
+def test_config1_full_vector_every_element():
+    """d = 2^20, n = 8, 20 steps: the whole state against the oracle, not a sample."""
+    w = synth.CONFIGS[1]
+    opt = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed)
+    ref32 = CSEROracle(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed, dtype=np.float32)
+    ref64 = CSEROracle(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed, dtype=np.float64)
+    x0 = synth.x0(w, DEV)
+    opt.set_x0(x0)
+    ref32.set_x0(x0.cpu().numpy()), ref64.set_x0(x0.cpu().numpy())
+    for t in range(1, w.steps + 1):
+        g = synth.gradients(w, t, DEV)
+        opt.step(g)
+        gh = g.cpu().numpy()
+        ref32.step(gh), ref64.step(gh)
+        assert np.array_equal(opt.state(b.STATE_MASK_G).cpu().numpy(), ref32.mask_g)
+        if t == 1:
+            for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e")):
+                assert _within(opt.state(which).cpu().numpy(), getattr(ref64, name), 1e-6, 1e-7).all()
+    for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e")):
+        got = opt.state(which).cpu().numpy()
+        want = getattr(ref64, name)
+        assert _within(got, want, 1e-4, 1e-4 * float(np.sqrt((want**2).mean()))).all()
+        assert np.array_equal(got, getattr(ref32, name))
+    with pytest.raises(b.CSERError):
+        opt.state(b.STATE_M)                       # no momentum array when beta == 0
+    opt.close()
+
+
+@pytest.mark.parametrize("cfg", [2, 3, 4])
+def test_full_size_configs_on_sampled_blocks(cfg):
+    _full_size_parity(cfg)
+
+
+def test_config5_bert_large_sized_on_sampled_blocks():
+    """About 43 GB of state and gradients; 64-bit indexing (n*d > 2^31)."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 70 * 2**30:
+        pytest.skip("needs about 65 GB of free device memory")
+    _full_size_parity(5, n_random=96)
+
+
+# ------------------------------------------------------------------ boundary behaviour
+def test_host_gradient_entry_point_equals_device_entry_point():
+    w = synth.CONFIGS[2].scaled(d=3_000_000 + 4, steps=10)
+    a = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, 5)
+    c = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, 5)
+    x0 = synth.x0(w, DEV)
+    a.set_x0(x0), c.set_x0(x0.cpu())             # x0 from device and from host memory
+    pinned = torch.empty((w.n_workers, w.d), dtype=torch.float32).pin_memory()
+    for t in range(1, w.steps + 1):
+        g = synth.gradients(w, t, DEV)
+        pinned.copy_(g)
+        a.step(g)
+        c.step_host(pinned)
+        torch.cuda.synchronize()
+    for which in (b.STATE_X, b.STATE_E, b.STATE_M, b.STATE_MASK_G, b.STATE_MASK_R):
+        assert torch.equal(a.state(which), c.state(which))
+    a.close(), c.close()
+
+
+def test_column_slabs_reproduce_the_whole_vector():
+    """Two handles that each own a slab of whole blocks, with global block ids, and exchange nothing."""
+    from paper_2007_13221_b200.shard import slab_of_rank
+    w = synth.CONFIGS[3].scaled(d=100_000 + 8, steps=9)
+    whole = b.CSER(w.d, w.n_workers, w.block_size, 4, 2, w.H, w.eta, w.beta, 1)
+    x0 = synth.x0(w, DEV)
+    whole.set_x0(x0)
+    slabs = []
+    for r in range(2):
+        c0, c1, b0 = slab_of_rank(w.d, w.block_size, r, 2)
+        s = b.CSER(c1 - c0, w.n_workers, w.block_size, 4, 2, w.H, w.eta, w.beta, 1, block_begin=b0)
+        s.set_x0(x0[c0:c1].contiguous())
+        slabs.append((c0, c1, s))
+    for t in range(1, w.steps + 1):
+        g = synth.gradients(w, t, DEV)
+        whole.step(g)
+        for c0, c1, s in slabs:
+            s.step(g[:, c0:c1].contiguous())
+    for which in (b.STATE_X, b.STATE_E, b.STATE_M):
+        full = whole.state(which)
+        for c0, c1, s in slabs:
+            assert torch.equal(full[:, c0:c1], s.state(which))
+    whole.close()
+    [s.close() for _, _, s in slabs]
+
+
+def test_checkpoint_and_resume_is_bit_identical():
+    w = synth.CONFIGS[2].scaled(d=50_000, steps=30)
+    a = b.CSER(w.d, w.n_workers, w.block_size, 4, 4, w.H, w.eta, w.beta, 2)
+    a.set_x0(synth.x0(w, DEV))
+    for t in range(1, 11):
+        a.step(synth.gradients(w, t, DEV))
+    snap = {k: a.state(k).clone() for k in (b.STATE_X, b.STATE_E, b.STATE_M)}
+    t_snap = a.t
+    for t in range(11, 21):
+        a.step(synth.gradients(w, t, DEV))
+    final = {k: a.state(k).clone() for k in (b.STATE_X, b.STATE_E, b.STATE_M)}
+    c = b.CSER(w.d, w.n_workers, w.block_size, 4, 4, w.H, w.eta, w.beta, 2)
+    for k, v in snap.items():
+        b.cser_write_state(c.h, k, v)
+    b.cser_write_state(c.h, b.STATE_T, torch.tensor([t_snap], dtype=torch.int64))
+    for t in range(11, 21):
+        c.step(synth.gradients(w, t, DEV))
+    for k in final:
+        assert torch.equal(final[k], c.state(k))
+    a.close(), c.close()
+
+
+def test_errors_are_reported_not_raised_on_the_device():
+    L = b.lib()
+    assert not L.cser_create(0, 8, 256, 4, 4, 4, 0.1, 0.0, 0)
+    assert "positive" in b.cser_last_error()
+    assert not L.cser_create(100, 8, 256, 0, 4, 4, 0.1, 0.0, 0)
+    assert not L.cser_create(100, 8, 256, 4, 4, 0, 0.1, 0.0, 0)
+    assert not L.cser_create(100, 8, 256, 4, 4, 4, float("nan"), 0.0, 0)
+    assert not L.cser_create(100, 8, 256, 4, 4, 4, 0.1, 1.0, 0)
+    assert L.cser_step(None, None, None) == -1
+    opt = b.CSER(100, 2, 10, 2, 2, 2, 0.1, 0.0, 0)
+    assert L.cser_step(opt.h, None, None) == -1
+    host = torch.zeros((2, 100))
+    assert L.cser_step(opt.h, ctypes.c_void_p(host.data_ptr()), None) == -1      # host pointer
+    assert "device memory" in b.cser_last_error()
+    small = torch.zeros(10, device=DEV)
+    assert L.cser_read_state(opt.h, b.STATE_X, ctypes.c_void_p(small.data_ptr()), 40, None) == -4
+    assert L.cser_read_state(opt.h, b.STATE_M, ctypes.c_void_p(small.data_ptr()), 40, None) == -1
+    assert L.cser_read_state(opt.h, 17, ctypes.c_void_p(small.data_ptr()), 40, None) == -1
+    assert opt.t == 0                                 # failed calls did not advance the step counter
+    opt.step(torch.zeros((2, 100), device=DEV))
+    assert opt.t == 1
+    opt.close()

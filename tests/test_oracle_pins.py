@@ -12,6 +12,8 @@ from fractions import Fraction
 import numpy as np
 import pytest
 
+from _golden import read_hand_example
+
 from oracle import (CSEROracle, CSERImpl2Oracle, grbs_mask, n_blocks, philox4_generic,
                     philox4x32_10, psync, STREAM_GRAD, STREAM_RESET)
 
@@ -205,21 +207,10 @@ def test_R1_with_momentum_is_nesterov_momentum_sgd_on_the_mean_gradient():
 
 
 # --------------------------------------------------------------------------- hand example
-def _read_golden():
-    rows = {}
-    with open(os.path.join(ROOT, "tests", "golden", "hand_example_n2_d4.txt")) as f:
-        for ln in f:
-            if ln.startswith("#") or not ln.strip():
-                continue
-            p = ln.split()
-            rows[(float(p[0]), int(p[1]), p[2], int(p[3]))] = [float(v) for v in p[4:]]
-    return rows
-
-
 @pytest.mark.parametrize("dtype", [np.float32, np.float64])
 @pytest.mark.parametrize("beta", [0.0, 0.5])
 def test_hand_worked_example(beta, dtype):
-    gold = _read_golden()
+    gold = read_hand_example()
     g = [np.array([[1, 2, -1, 0], [3, -2, 1, 4]], np.float32), np.array([[2, 2, 2, 2], [0, 4, -2, 6]], np.float32)]
     masks = [([1, 0], None), ([0, 1], [0, 1])]
     o = CSEROracle(4, 2, 2, 7, 7, 2, 0.5, beta, 0, dtype=dtype)
