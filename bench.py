@@ -177,11 +177,14 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--ring", type=int, default=0, help="distinct gradient buffers cycled through")
+    ap.add_argument("--d", type=int, default=0, help="override the vector length (small profiling cases)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
     from paper_2007_13221_b200 import synth
     w = synth.CONFIGS[args.config]
+    if args.d:
+        w = w.scaled(args.d)
     if args.impl == "reference":
         run_reference(args, w)
         return
