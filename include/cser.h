@@ -169,6 +169,42 @@ int cser_last_kernel_ms(cser_handle h, float *mask_ms, float *step_ms);
 /* Number of kernels this library has launched on behalf of the handle. */
 int64_t cser_launch_count(cser_handle h);
 
+/*
+ * One iteration without any allocation (the paper has no counterpart: this is a
+ * calling convenience of this library, not a part of the algorithm).
+ *
+ * Who it is for: code that may not call cudaMalloc at the point where it steps the
+ * optimizer - a host framework that owns all device memory through its own pool and
+ * forbids driver allocations once training runs (cudaMalloc can stall every stream of
+ * the device), a real-time loop that must not take the allocator's locks, or a plug-in
+ * that is handed its buffers and has no right to create state of its own.  Such a
+ * caller owns x, e and m itself (device, fp32 [n, d] row-major, updated in place) and
+ * keeps the step counter; cser_create is never called and nothing has to be destroyed.
+ *
+ * It performs exactly the iteration `t` (1-based; resets when t mod H == 0) that
+ * cser_step performs on a handle whose counter stands at t - 1, with the same kernels
+ * and the same arithmetic.  m is ignored (may be NULL) when beta == 0.
+ *
+ * Scratch: the two GRBS masks are kept in a fixed array inside the library, in the
+ * device memory of every GPU that loads it, for the life of the process
+ * (2 * CSER_NOALLOC_MAX_BLOCKS bytes = 512 KiB per GPU).  A vector with more than
+ * CSER_NOALLOC_MAX_BLOCKS blocks (ceil(d / block_size)) is refused with
+ * CSER_ERR_INVALID; choose a larger block_size or use the handle API.
+ *
+ * The first call on each device looks up the array's device address (no allocation,
+ * but a runtime query); make that first call outside any stream capture.
+ * All calls on a device share the one array: the masks of a call are overwritten by
+ * the next.  Each call rewrites every mask entry it later reads, so no clearing is
+ * needed between calls, but two calls whose kernels may overlap on the GPU (different
+ * streams, or different host threads) race on the masks - serialize them on one stream.
+ * No cudaMalloc, cudaFree or other allocating routine is called.
+ */
+#define CSER_NOALLOC_MAX_BLOCKS 262144
+int cser_step_noalloc(int64_t d, int32_t n_workers, int32_t block_size,
+                      uint32_t R1, uint32_t R2, int32_t H,
+                      float eta, float beta, uint64_t seed, uint64_t t,
+                      const float *grad, float *x, float *e, float *m, void *stream);
+
 /* Thread-local description of the last error in this thread ("" if none). */
 const char *cser_last_error(void);
 

@@ -51,6 +51,10 @@ def lib():
     L.cser_last_kernel_ms.argtypes = [c.c_void_p, c.POINTER(c.c_float), c.POINTER(c.c_float)]
     L.cser_launch_count.restype = c.c_int64
     L.cser_launch_count.argtypes = [c.c_void_p]
+    L.cser_step_noalloc.restype = c.c_int
+    L.cser_step_noalloc.argtypes = [c.c_int64, c.c_int32, c.c_int32, c.c_uint32, c.c_uint32, c.c_int32,
+                                    c.c_float, c.c_float, c.c_uint64, c.c_uint64,
+                                    c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
     L.cser_last_error.restype = c.c_char_p
     L.cser_last_error.argtypes = []
     for name in ("cser_set_x0", "cser_step", "cser_step_host", "cser_read_state", "cser_write_state",
@@ -122,6 +126,13 @@ def cser_debug_set_masks(h, g_mask, r_mask=None, stream=None):
 def cser_grbs_mask(seed, t, which, block_begin, n_blocks, R, mask_out, stream=None):
     _check(lib().cser_grbs_mask(seed, t, which, block_begin, n_blocks, R, _ptr(mask_out), _stream(stream)),
            "cser_grbs_mask")
+
+
+def cser_step_noalloc(d, n_workers, block_size, R1, R2, H, eta, beta, seed, t, grad, x, e, m=None, stream=None):
+    """One iteration t on arrays the caller owns; the library allocates nothing (see cser.h)."""
+    _check(lib().cser_step_noalloc(d, n_workers, block_size, R1, R2, H, eta, beta, seed, t, _ptr(grad),
+                                   _ptr(x), _ptr(e), _ptr(m) if m is not None else None, _stream(stream)),
+           "cser_step_noalloc")
 
 
 def cser_set_timing(h, on):

@@ -658,3 +658,81 @@ int cser_last_kernel_ms(cser_handle h, float *mask_ms, float *step_ms) {
 int64_t cser_launch_count(cser_handle h) { return h ? h->launches : 0; }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------ allocation-free step
+// The two GRBS masks are the only scratch memory a step needs.  For callers that must
+// not allocate, they live here: a fixed array that every GPU which loads this library
+// keeps until the process exits (2 * CSER_NOALLOC_MAX_BLOCKS bytes).  The first half
+// holds the update mask, the second half the reset mask.
+static __device__ __align__(256) uint8_t g_noalloc_masks[2 * CSER_NOALLOC_MAX_BLOCKS];
+
+namespace {
+
+constexpr int kNoallocMaxDevices = 64;
+// Device address of g_noalloc_masks on each device, looked up once per device.  In host
+// code the array's name is only a handle for the runtime, never an address a kernel may
+// be given; cudaGetSymbolAddress translates it for the device that is current.
+uint8_t *g_noalloc_addr[kNoallocMaxDevices] = {};
+
+int noalloc_scratch(int device, uint8_t **out) {
+    if (device < 0 || device >= kNoallocMaxDevices)
+        return fail(CSER_ERR_INVALID, "cser_step_noalloc: device %d out of range", device);
+    uint8_t *p = __atomic_load_n(&g_noalloc_addr[device], __ATOMIC_ACQUIRE);
+    if (!p) {
+        void *sym = nullptr;
+        cudaError_t er = cudaGetSymbolAddress(&sym, g_noalloc_masks);
+        if (er != cudaSuccess || !sym) {
+            cudaGetLastError();
+            return fail(CSER_ERR_CUDA, "cser_step_noalloc: cudaGetSymbolAddress: %s",
+                        cudaGetErrorString(er));
+        }
+        p = static_cast<uint8_t *>(sym);
+        __atomic_store_n(&g_noalloc_addr[device], p, __ATOMIC_RELEASE);
+    }
+    *out = p;
+    return CSER_OK;
+}
+
+}  // namespace
+
+extern "C" int cser_step_noalloc(int64_t d, int32_t n_workers, int32_t block_size, uint32_t R1,
+                                 uint32_t R2, int32_t H, float eta, float beta, uint64_t seed,
+                                 uint64_t t, const float *grad, float *x, float *e, float *m,
+                                 void *stream) {
+    if (d <= 0 || n_workers <= 0 || block_size <= 0 || R1 == 0 || R2 == 0 || H <= 0 || t == 0)
+        return fail(CSER_ERR_INVALID,
+                    "cser_step_noalloc: d, n_workers, block_size, R1, R2, H, t must be positive");
+    if (!isfinite(eta) || !(beta >= 0.f && beta < 1.f))
+        return fail(CSER_ERR_INVALID, "cser_step_noalloc: eta must be finite and beta in [0, 1)");
+    const long long B = (d + block_size - 1) / block_size;
+    if (B > (long long)CSER_NOALLOC_MAX_BLOCKS)
+        return fail(CSER_ERR_INVALID,
+                    "cser_step_noalloc: %lld blocks exceed the built-in scratch of %d blocks; "
+                    "use a larger block_size or the handle API", B, (int)CSER_NOALLOC_MAX_BLOCKS);
+    if (int rc = check_device_ptr(grad, "cser_step_noalloc: grad")) return rc;
+    if (int rc = check_device_ptr(x, "cser_step_noalloc: x")) return rc;
+    if (int rc = check_device_ptr(e, "cser_step_noalloc: e")) return rc;
+    if (beta != 0.f) {
+        if (int rc = check_device_ptr(m, "cser_step_noalloc: m")) return rc;
+    }
+    if (((uintptr_t)grad | (uintptr_t)x | (uintptr_t)e | (uintptr_t)m) % 4 != 0)
+        return fail(CSER_ERR_INVALID, "cser_step_noalloc: arrays must be 4-byte aligned");
+
+    cser_ctx c;   // plain stack object describing the caller's arrays; owns nothing
+    CU_TRY(cudaGetDevice(&c.device));
+    uint8_t *masks = nullptr;
+    if (int rc = noalloc_scratch(c.device, &masks)) return rc;
+    c.d = d, c.n = n_workers, c.bs = block_size, c.R1 = R1, c.R2 = R2, c.H = H;
+    c.eta = eta, c.beta = beta, c.seed = seed, c.B = B, c.block_begin = 0;
+    c.t = t;
+    c.x = x, c.e = e, c.m = (beta != 0.f) ? m : nullptr;
+    c.mask_g = masks, c.mask_r = masks + CSER_NOALLOC_MAX_BLOCKS;
+    c.vec4 = (d % 4 == 0) && (block_size % 4 == 0) &&
+             (((uintptr_t)x | (uintptr_t)e | (uintptr_t)c.m) % 16 == 0);
+    const bool is_reset = (t % (uint64_t)H) == 0;
+    cudaStream_t s = (cudaStream_t)stream;
+    // Both masks are rewritten for all B blocks before the step kernel reads them, so
+    // nothing left in the array by an earlier call is ever used.
+    if (int rc = launch_masks(&c, is_reset, s)) return rc;
+    return launch_step(&c, grad, 0, d, is_reset, s);
+}

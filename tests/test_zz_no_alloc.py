@@ -1,0 +1,54 @@
+"""The allocation-free entry point against the handle-based one.
+
+Some callers cannot call cudaMalloc where they step the optimizer (all device memory
+belongs to their framework's pool, or an allocation would stall their other streams).
+cser_step_noalloc serves them: the caller owns x, e, m and the step counter, and the
+masks live in a fixed array inside the library.  This file is named so that pytest
+collects it last; it must pass alone in a fresh process and after all other tests.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2007_13221_b200 import binding as b, synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.mark.parametrize("beta,d", [(0.9, 200_000 + 36), (0.0, 50_001)])
+def test_noalloc_step_equals_handle_step_on_consecutive_calls(beta, d):
+    import __graft_entry__
+    __graft_entry__.build()
+    torch.cuda.set_device(0)
+    w = synth.CONFIGS[2].scaled(d=d, steps=6)
+    n, bs, R1, R2, H, eta, seed = w.n_workers, w.block_size, 4, 2, 2, w.eta, 11
+    ref = b.CSER(d, n, bs, R1, R2, H, eta, beta, seed)
+    x0 = synth.x0(w, DEV)
+    ref.set_x0(x0)
+    x = x0[None, :].repeat(n, 1).contiguous()
+    e = torch.zeros_like(x)
+    m = torch.zeros_like(x) if beta else None
+    for t in range(1, w.steps + 1):                # t = 2, 4, 6 are reset steps
+        g = synth.gradients(w, t, DEV)
+        ref.step(g)
+        b.cser_step_noalloc(d, n, bs, R1, R2, H, eta, beta, seed, t, g, x, e, m)
+        torch.cuda.synchronize()
+        # same tolerance as the other GPU tests use between identical arithmetic: exact
+        assert torch.equal(ref.state(b.STATE_X), x), t
+        assert torch.equal(ref.state(b.STATE_E), e), t
+        if beta:
+            assert torch.equal(ref.state(b.STATE_M), m), t
+    ref.close()
+
+
+def test_noalloc_rejects_vectors_beyond_its_built_in_scratch():
+    torch.cuda.set_device(0)
+    L = b.lib()
+    max_blocks = 262144
+    z = torch.zeros(8, device=DEV)
+    rc = L.cser_step_noalloc((max_blocks + 1) * 4, 1, 4, 2, 2, 2, 0.1, 0.0, 0, 1,
+                             z.data_ptr(), z.data_ptr(), z.data_ptr(), None, None)
+    assert rc == -1 and "exceed" in b.cser_last_error()
+    rc = L.cser_step_noalloc(8, 1, 4, 2, 2, 2, 0.1, 0.0, 0, 0, z.data_ptr(), z.data_ptr(), z.data_ptr(), None, None)
+    assert rc == -1                                 # t is 1-based
