@@ -185,18 +185,19 @@ int64_t cser_launch_count(cser_handle h);
  * cser_step performs on a handle whose counter stands at t - 1, with the same kernels
  * and the same arithmetic.  m is ignored (may be NULL) when beta == 0.
  *
- * Scratch: the two GRBS masks are kept in a fixed array inside the library, in the
- * device memory of every GPU that loads it, for the life of the process
- * (2 * CSER_NOALLOC_MAX_BLOCKS bytes = 512 KiB per GPU).  A vector with more than
+ * Scratch: the two GRBS masks and the list of selected blocks are kept in a fixed array
+ * inside the library, in the device memory of every GPU that loads it, for the life of
+ * the process (6 * CSER_NOALLOC_MAX_BLOCKS + 256 bytes = 1.5 MiB per GPU).  A vector with more than
  * CSER_NOALLOC_MAX_BLOCKS blocks (ceil(d / block_size)) is refused with
  * CSER_ERR_INVALID; choose a larger block_size or use the handle API.
  *
  * The first call on each device looks up the array's device address (no allocation,
  * but a runtime query); make that first call outside any stream capture.
- * All calls on a device share the one array: the masks of a call are overwritten by
- * the next.  Each call rewrites every mask entry it later reads, so no clearing is
- * needed between calls, but two calls whose kernels may overlap on the GPU (different
- * streams, or different host threads) race on the masks - serialize them on one stream.
+ * All calls on a device share the one array: the masks and list of a call are
+ * overwritten by the next.  Each call rewrites every entry it later reads and clears the
+ * list counter the following call will use, so no clearing is needed between calls, but
+ * two calls whose kernels may overlap on the GPU (different streams, or different host
+ * threads) race on the array - serialize them on one stream and one host thread.
  * No cudaMalloc, cudaFree or other allocating routine is called.
  */
 #define CSER_NOALLOC_MAX_BLOCKS 262144

@@ -1,13 +1,16 @@
 // CSER / M-CSER optimizer step for B200 (sm_100a): GRBS mask kernel, fused step
 // kernel and the C ABI declared in include/cser.h.
 //
-// Layout: g, x, e, m are fp32 [n, d] row-major (worker-major).  A thread owns one
-// vector column (4 consecutive elements, or 1 in the scalar fallback) and walks
-// the worker axis, so every warp access is a contiguous 512-byte run of one row.
-// The step is bound by HBM traffic (about 28 bytes per element and worker against
-// 7 flops), so the kernel is organised around keeping many independent 16-byte
-// loads in flight per thread and touching every byte exactly once; there is no
-// contraction here and tensor cores are not used.
+// Layout: g, x, e, m are fp32 [n, d] row-major (worker-major).  The step is bound
+// by HBM traffic (about 28 bytes per element and worker against 7 flops), so the
+// kernel is organised around how DRAM likes to be walked: the grid is (column
+// tiles, workers) and CTAs are dispatched tile-fastest, so the unselected blocks
+// (all but 1/R of the data, purely elementwise) are streamed row after row as four
+// long contiguous read streams and three write streams, every byte touched once.
+// Blocks selected by a mask (1/R of the data) need the mean over workers: an extra
+// row of CTAs, dispatched first, handles them with 8 worker lanes per column that
+// meet in shared memory.  There is no contraction here and tensor cores are not
+// used.
 //
 // Compiled with -fmad=false: every multiply and add rounds separately, in the
 // order stated in include/cser.h.
@@ -79,6 +82,45 @@ grbs_mask_kernel(uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r, lon
     (second ? mask_r : mask_g)[b] = sel;
 }
 
+// Per-step block select: one thread per block.  With `draw` it draws the update mask (and,
+// on a reset step, the reset mask) and stores the flags; without it the flags already in
+// mask_g / mask_r are used (injected masks).  Blocks selected by either mask are appended
+// to `list` (order irrelevant: blocks are independent) with one atomicAdd per warp on
+// *count.  *count_next, the counter the following step will use, is cleared here, so no
+// counter ever needs a separate memset.
+__global__ void __launch_bounds__(256)
+grbs_select_kernel(uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r,
+                   uint32_t *__restrict__ list, uint32_t *count, uint32_t *count_next, long long B,
+                   long long block_begin, uint32_t k0, uint32_t k1, uint32_t t_lo, uint32_t t_hi,
+                   uint32_t R_g, uint32_t R_r, int is_reset, int draw) {
+    const long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (b == 0) *count_next = 0;
+    bool sg = false, sr = false;
+    if (b < B) {
+        if (draw) {
+            const uint32_t gb = (uint32_t)(block_begin + b);
+            sg = (unsigned long long)philox4x32_10_word0(k0, k1, gb, t_lo, t_hi, 0u) * R_g < (1ull << 32);
+            mask_g[b] = sg ? 1 : 0;
+            if (is_reset) {
+                sr = (unsigned long long)philox4x32_10_word0(k0, k1, gb, t_lo, t_hi, 1u) * R_r < (1ull << 32);
+                mask_r[b] = sr ? 1 : 0;
+            }
+        } else {
+            sg = mask_g[b] != 0;
+            sr = is_reset ? (mask_r[b] != 0) : false;
+        }
+    }
+    const bool need = sg || sr;
+    const unsigned ballot = __ballot_sync(0xffffffffu, need);
+    if (ballot == 0) return;
+    const unsigned lane = threadIdx.x & 31;
+    const int leader = __ffs(ballot) - 1;
+    unsigned base = 0;
+    if ((int)lane == leader) base = atomicAdd(count, (unsigned)__popc(ballot));
+    base = __shfl_sync(0xffffffffu, base, leader);
+    if (need) list[base + __popc(ballot & ((1u << lane) - 1u))] = (uint32_t)b;
+}
+
 // ------------------------------------------------------------------ fused step
 template <int V>
 struct Pack {
@@ -123,10 +165,15 @@ struct StepParams {
     const float *g;
     float *x, *e, *m;
     const uint8_t *mask_g, *mask_r;
-    long long d;         // elements per row
-    long long c_begin;   // first vector column handled by this launch
-    long long c_end;     // one past the last
-    unsigned bsv;        // GRBS block size in vector columns
+    const uint32_t *list;    // blocks selected by either mask this step
+    const uint32_t *count;   // how many
+    long long d;             // elements per row
+    long long cols_total;    // vector columns per row
+    long long c_begin;       // first vector column handled by this launch
+    long long c_end;         // one past the last
+    unsigned bsv;            // GRBS block size in vector columns
+    unsigned tiles;          // tiles of 256 vector columns in [c_begin, c_end)
+    unsigned sel_ctas;       // leading CTAs of the grid that work on the selected blocks
     int n;
     float eta, beta, n_f;
 };
@@ -149,138 +196,212 @@ __device__ __forceinline__ Pack<V> get_p(const Pack<V> &g, Pack<V> &m, float eta
     return p;
 }
 
-// One thread = one vector column, all workers.  U = workers whose loads are
-// issued together before any of their results is used.
-template <int V, bool MOM, bool RESET, int U>
-__global__ void __launch_bounds__(256) cser_step_kernel(const StepParams P) {
-    const long long c = P.c_begin + (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (c >= P.c_end) return;
-    const long long b = (P.c_end <= 0xffffffffll) ? (long long)((uint32_t)c / P.bsv)
-                                                  : (long long)((unsigned long long)c / P.bsv);
-    const bool sg = P.mask_g[b] != 0;
-    const bool sr = RESET ? (P.mask_r[b] != 0) : false;
+// Shape of the CTA that handles selected columns: 32 vector columns x 8 worker lanes.
+constexpr int kSelCols = 32;
+constexpr int kSelLanes = 8;
+constexpr int kStepThreads = kSelCols * kSelLanes;   // 256
+#ifndef CSER_SEL_CTAS_PER_SM
+#define CSER_SEL_CTAS_PER_SM 4
+#endif
+constexpr int kSelCtasPerSm = CSER_SEL_CTAS_PER_SM;  // CTAs per SM given to the selected blocks
+
+// Ordered sum over the workers of one lane chunk: acc = ((acc + S[0]) + S[1]) + ...,
+// starting from S[0] itself when `first` (no 0.0f is ever added).
+template <int V>
+__device__ __forceinline__ void ordered_accumulate(Pack<V> &acc, const Pack<V> (*S)[kSelCols], int cv,
+                                                   int cnt, bool first) {
+    for (int k = 0; k < cnt; ++k) {
+        const Pack<V> s = S[k][cv];
+#pragma unroll
+        for (int q = 0; q < V; ++q) acc.v[q] = (first && k == 0) ? s.v[q] : acc.v[q] + s.v[q];
+    }
+}
+
+// Selected blocks, all workers.  The first P.sel_ctas CTAs of the grid share the list of
+// selected blocks in pieces of at most 256 vector columns.  A piece is walked in chunks of
+// 32 columns; in a chunk, warp w owns worker lane w, so every access is one contiguous run
+// of a row, and the workers' values of a column meet in shared memory, where they are
+// summed in ascending worker order.  A block's two mask flags are uniform over the CTA.
+template <int V, bool MOM, bool RESET>
+__device__ __forceinline__ void selected_blocks_role(const StepParams &P) {
+    __shared__ Pack<V> S[2][kSelLanes][kSelCols];
+    const int cv = threadIdx.x & (kSelCols - 1);
+    const int wl = threadIdx.x / kSelCols;
     const long long d = P.d;
     const int n = P.n;
     const float eta = P.eta, beta = P.beta;
-    const float *__restrict__ g = P.g + c * V;
-    float *__restrict__ x = P.x + c * V;
-    float *__restrict__ e = P.e + c * V;
-    float *__restrict__ m = MOM ? P.m + c * V : nullptr;
+    const unsigned pieces_per_block = (P.bsv + kStepThreads - 1) / kStepThreads;
+    const unsigned long long items = (unsigned long long)(*P.count) * pieces_per_block;
+    int buf = 0;
 
-    if (!sg && !sr) {
-        // Unselected block, no reset: C(p) = 0, so p' = r = p (Algorithm 3 lines 4-8):
-        // x_i -= p_i, e_i -= p_i.  Purely elementwise.
-        for (int i0 = 0; i0 < n; i0 += U) {
-            Pack<V> gv[U], mv[U], xv[U], ev[U];
+    for (unsigned long long w = blockIdx.x; w < items; w += P.sel_ctas) {
+        const unsigned blk = P.list[w / pieces_per_block];
+        const unsigned piece = (unsigned)(w % pieces_per_block);
+        const bool sg = P.mask_g[blk] != 0;
+        const bool sr = RESET ? (P.mask_r[blk] != 0) : false;
+        const bool only_r = sr && !sg;
+        const long long blk_c0 = (long long)blk * P.bsv;
+        long long c_lo = blk_c0 + (long long)piece * kStepThreads;
+        long long c_hi = min(min(c_lo + kStepThreads, blk_c0 + (long long)P.bsv), P.cols_total);
+        c_lo = max(c_lo, P.c_begin);
+        c_hi = min(c_hi, P.c_end);
+
+        for (long long cc = c_lo; cc < c_hi; cc += kSelCols) {
+            const long long c = cc + cv;
+            const bool valid = c < c_hi;
+            const float *__restrict__ g = P.g + c * V;
+            float *__restrict__ x = P.x + c * V;
+            float *__restrict__ e = P.e + c * V;
+            float *__restrict__ m = MOM ? P.m + c * V : nullptr;
+            Pack<V> sum_p, sum_e;
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                if (i0 + u < n) {
-                    const long long o = (long long)(i0 + u) * d;
-                    gv[u] = ld_stream<V>(g + o);
-                    if constexpr (MOM) mv[u] = ld<V>(m + o);
-                    xv[u] = ld<V>(x + o);
-                    ev[u] = ld<V>(e + o);
+            for (int q = 0; q < V; ++q) sum_p.v[q] = sum_e.v[q] = 0.f;
+
+            // The first round's x (and e) of an update-selected block are fetched together
+            // with its g and m, so that a chunk costs one memory round trip, not two.
+            Pack<V> x0v, e0v;
+#pragma unroll
+            for (int q = 0; q < V; ++q) x0v.v[q] = e0v.v[q] = 0.f;
+            if (sg && valid && wl < n) {
+                x0v = ld<V>(x + (long long)wl * d);
+                if (sr) e0v = ld<V>(e + (long long)wl * d);
+            }
+
+            // Pass 1: Get_p for every worker.  An update-selected block gathers sum_k p_k.
+            // A block selected by the reset mask only takes its own residual step here
+            // (x_{t-1/2} = x - p, e_{t-1/2} = e - p), stores x_{t-1/2} - e_{t-1/2}, zeroes
+            // e and gathers sum_k e_{k,t-1/2}.
+            for (int i0 = 0; i0 < n; i0 += kSelLanes) {
+                const int i = i0 + wl;
+                const long long o = (long long)i * d;
+                Pack<V> p, eh;
+#pragma unroll
+                for (int q = 0; q < V; ++q) p.v[q] = eh.v[q] = 0.f;
+                if (valid && i < n) {
+                    const Pack<V> gv = ld_stream<V>(g + o);
+                    Pack<V> mv, xv, ev;
+                    if constexpr (MOM) mv = ld<V>(m + o);
+                    if (only_r) {
+                        xv = ld<V>(x + o);
+                        ev = ld<V>(e + o);
+                    }
+                    p = get_p<V, MOM>(gv, mv, eta, beta);
+                    if constexpr (MOM) st<V>(m + o, mv);
+                    if (only_r) {
+                        Pack<V> z;
+#pragma unroll
+                        for (int q = 0; q < V; ++q) {
+                            const float xh = xv.v[q] - p.v[q];
+                            eh.v[q] = ev.v[q] - p.v[q];
+                            xv.v[q] = xh - eh.v[q];
+                            z.v[q] = 0.f;
+                        }
+                        st<V>(x + o, xv);
+                        st<V>(e + o, z);
+                    }
+                }
+                S[buf][wl][cv] = only_r ? eh : p;
+                __syncthreads();
+                ordered_accumulate<V>(only_r ? sum_e : sum_p, S[buf], cv, min(kSelLanes, n - i0), i0 == 0);
+                buf ^= 1;                                // the next round writes the other buffer
+            }
+
+            // Pass 2 (update-selected block): x_i -= mean_k p_k; e untouched.  If the block is
+            // reset-selected too: store (x_i - p-bar) - e_i, zero e, gather sum_k e_k.
+            if (sg) {
+                Pack<V> pbar;
+#pragma unroll
+                for (int q = 0; q < V; ++q) pbar.v[q] = sum_p.v[q] / P.n_f;
+                for (int i0 = 0; i0 < n; i0 += kSelLanes) {
+                    const int i = i0 + wl;
+                    const long long o = (long long)i * d;
+                    Pack<V> ev;
+#pragma unroll
+                    for (int q = 0; q < V; ++q) ev.v[q] = 0.f;
+                    if (valid && i < n) {
+                        Pack<V> xv = x0v;
+                        if (i0 == 0) {
+                            ev = e0v;
+                        } else {
+                            xv = ld<V>(x + o);
+                            if (sr) ev = ld<V>(e + o);
+                        }
+#pragma unroll
+                        for (int q = 0; q < V; ++q) xv.v[q] = xv.v[q] - pbar.v[q];
+                        if (sr) {
+                            Pack<V> z;
+#pragma unroll
+                            for (int q = 0; q < V; ++q) {
+                                xv.v[q] = xv.v[q] - ev.v[q];
+                                z.v[q] = 0.f;
+                            }
+                            st<V>(e + o, z);
+                        }
+                        st<V>(x + o, xv);
+                    }
+                    if (sr) {
+                        S[buf][wl][cv] = ev;
+                        __syncthreads();
+                        ordered_accumulate<V>(sum_e, S[buf], cv, min(kSelLanes, n - i0), i0 == 0);
+                        buf ^= 1;
+                    }
                 }
             }
+
+            // Pass 3 (reset-selected block), Algorithm 2 lines 11-12:
+            // x_i = (x_{i,t-1/2} - e_{i,t-1/2}) + mean_k e_{k,t-1/2}.
+            if (sr && valid) {
+                Pack<V> ebar;
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                if (i0 + u < n) {
-                    const long long o = (long long)(i0 + u) * d;
-                    const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], eta, beta);
+                for (int q = 0; q < V; ++q) ebar.v[q] = sum_e.v[q] / P.n_f;
+                for (int i = wl; i < n; i += kSelLanes) {
+                    const long long o = (long long)i * d;
+                    Pack<V> xv = ld<V>(x + o);
 #pragma unroll
-                    for (int k = 0; k < V; ++k) {
-                        xv[u].v[k] = xv[u].v[k] - p.v[k];
-                        ev[u].v[k] = ev[u].v[k] - p.v[k];
-                    }
-                    if constexpr (MOM) st<V>(m + o, mv[u]);
-                    st<V>(x + o, xv[u]);
-                    st<V>(e + o, ev[u]);
+                    for (int q = 0; q < V; ++q) xv.v[q] = xv.v[q] + ebar.v[q];
+                    st<V>(x + o, xv);
                 }
             }
         }
+    }
+}
+
+// 1-D grid.  CTAs [0, sel_ctas), dispatched first, work on the selected blocks.  CTA
+// sel_ctas + i * tiles + tile streams tile `tile` of worker i: thread t owns vector column
+// c = c_begin + 256 * tile + t and updates it element by element unless a mask selects
+// its block.  Consecutive CTAs walk one row after the other, contiguously.
+template <int V, bool MOM, bool RESET>
+__global__ void __launch_bounds__(kStepThreads, 8) cser_step_kernel(const StepParams P) {
+    if (blockIdx.x < P.sel_ctas) {
+        selected_blocks_role<V, MOM, RESET>(P);
         return;
     }
-
-    Pack<V> sum_e;   // sum over workers of e_{t-1/2} (reset-selected columns)
+    const unsigned id = blockIdx.x - P.sel_ctas;
+    const unsigned row = id / P.tiles;
+    const unsigned tile = id - row * P.tiles;
+    const long long c = P.c_begin + (long long)tile * kStepThreads + threadIdx.x;
+    if (c >= P.c_end) return;
+    const long long b = (P.c_end <= 0xffffffffll) ? (long long)((uint32_t)c / P.bsv)
+                                                  : (long long)((unsigned long long)c / P.bsv);
+    if (P.mask_g[b] != 0) return;
+    if (RESET && P.mask_r[b] != 0) return;
+    // Unselected block, no reset: C(p) = 0, so p' = r = p (Algorithm 3 lines 4-8):
+    // x_i -= p_i, e_i -= p_i.  Purely elementwise.
+    const long long o = (long long)row * P.d + c * V;
+    const Pack<V> gv = ld_stream<V>(P.g + o);
+    Pack<V> mv;
+    if constexpr (MOM) mv = ld<V>(P.m + o);
+    Pack<V> xv = ld<V>(P.x + o);
+    Pack<V> ev = ld<V>(P.e + o);
+    const Pack<V> p = get_p<V, MOM>(gv, mv, P.eta, P.beta);
 #pragma unroll
-    for (int k = 0; k < V; ++k) sum_e.v[k] = 0.f;
-
-    if (sg) {
-        // Selected block: r = 0, p' = mean_k p_k.  Pass A forms the mean (and updates m).
-        Pack<V> sum_p;
-#pragma unroll
-        for (int k = 0; k < V; ++k) sum_p.v[k] = 0.f;
-        for (int i = 0; i < n; ++i) {
-            const long long o = (long long)i * d;
-            const Pack<V> gv = ld_stream<V>(g + o);
-            Pack<V> mv;
-            if constexpr (MOM) mv = ld<V>(m + o);
-            const Pack<V> p = get_p<V, MOM>(gv, mv, eta, beta);
-            if constexpr (MOM) st<V>(m + o, mv);
-#pragma unroll
-            for (int k = 0; k < V; ++k) sum_p.v[k] = (i == 0) ? p.v[k] : sum_p.v[k] + p.v[k];
-        }
-        Pack<V> pbar;
-#pragma unroll
-        for (int k = 0; k < V; ++k) pbar.v[k] = sum_p.v[k] / P.n_f;
-        // Pass B: x_i -= p-bar.  On a reset-selected column also fold in x - e and zero e.
-        for (int i = 0; i < n; ++i) {
-            const long long o = (long long)i * d;
-            Pack<V> xv = ld<V>(x + o);
-#pragma unroll
-            for (int k = 0; k < V; ++k) xv.v[k] = xv.v[k] - pbar.v[k];
-            if (sr) {
-                const Pack<V> ev = ld<V>(e + o);
-                Pack<V> z;
-#pragma unroll
-                for (int k = 0; k < V; ++k) {
-                    sum_e.v[k] = (i == 0) ? ev.v[k] : sum_e.v[k] + ev.v[k];
-                    xv.v[k] = xv.v[k] - ev.v[k];
-                    z.v[k] = 0.f;
-                }
-                st<V>(e + o, z);
-            }
-            st<V>(x + o, xv);
-        }
-    } else {
-        // Unselected by the update mask but reset-selected: x_{t-1/2} = x - p,
-        // e_{t-1/2} = e - p; store x_{t-1/2} - e_{t-1/2}, accumulate e_{t-1/2}, zero e.
-        for (int i = 0; i < n; ++i) {
-            const long long o = (long long)i * d;
-            const Pack<V> gv = ld_stream<V>(g + o);
-            Pack<V> mv;
-            if constexpr (MOM) mv = ld<V>(m + o);
-            Pack<V> xv = ld<V>(x + o);
-            const Pack<V> ev = ld<V>(e + o);
-            const Pack<V> p = get_p<V, MOM>(gv, mv, eta, beta);
-            if constexpr (MOM) st<V>(m + o, mv);
-            Pack<V> z;
-#pragma unroll
-            for (int k = 0; k < V; ++k) {
-                const float xh = xv.v[k] - p.v[k];
-                const float eh = ev.v[k] - p.v[k];
-                sum_e.v[k] = (i == 0) ? eh : sum_e.v[k] + eh;
-                xv.v[k] = xh - eh;
-                z.v[k] = 0.f;
-            }
-            st<V>(x + o, xv);
-            st<V>(e + o, z);
-        }
+    for (int k = 0; k < V; ++k) {
+        xv.v[k] = xv.v[k] - p.v[k];
+        ev.v[k] = ev.v[k] - p.v[k];
     }
-
-    if (sr) {
-        // Error reset (Algorithm 2 lines 11-12): x_i = (x_{t-1/2} - e_{t-1/2}) + mean_k e_k.
-        Pack<V> ebar;
-#pragma unroll
-        for (int k = 0; k < V; ++k) ebar.v[k] = sum_e.v[k] / P.n_f;
-        for (int i = 0; i < n; ++i) {
-            const long long o = (long long)i * d;
-            Pack<V> xv = ld<V>(x + o);
-#pragma unroll
-            for (int k = 0; k < V; ++k) xv.v[k] = xv.v[k] + ebar.v[k];
-            st<V>(x + o, xv);
-        }
-    }
+    if constexpr (MOM) st<V>(P.m + o, mv);
+    st<V>(P.x + o, xv);
+    st<V>(P.e + o, ev);
 }
 
 // x_i <- x0 for all workers; e, m <- 0
@@ -309,6 +430,10 @@ struct cser_ctx {
     uint64_t seed = 0, t = 0;
     float *x = nullptr, *e = nullptr, *m = nullptr;
     uint8_t *mask_g = nullptr, *mask_r = nullptr;
+    uint32_t *sel_list = nullptr;                    // [B] blocks selected this step
+    uint32_t *sel_count = nullptr;                   // [2] counters, used alternately
+    int flip = 0;                                    // which counter the next step uses
+    int sel_ctas = 0;                                // CTAs of the step kernel given to selected blocks
     float *x0_stage = nullptr;                       // [d] staging for a host x0
     bool masks_injected = false;
     bool vec4 = false;                               // 128-bit path usable for the state arrays
@@ -327,33 +452,37 @@ namespace {
 
 size_t state_elems(const cser_ctx *h) { return (size_t)h->n * (size_t)h->d; }
 
-int launch_masks(cser_ctx *h, bool is_reset, cudaStream_t s) {
-    const int n_masks = is_reset ? 2 : 1;
-    const long long total = h->B * n_masks;
-    const unsigned grid = (unsigned)((total + 255) / 256);
-    grbs_mask_kernel<<<grid, 256, 0, s>>>(h->mask_g, h->mask_r, h->B, h->block_begin,
-                                          (uint32_t)(h->seed & 0xffffffffu), (uint32_t)(h->seed >> 32),
-                                          (uint32_t)(h->t & 0xffffffffu), (uint32_t)(h->t >> 32),
-                                          h->R1, h->R2, n_masks, 0u);
+// GRBS select kernel of iteration h->t.  Leaves the step's counter index in h->flip ^ 1.
+int launch_select(cser_ctx *h, bool is_reset, bool draw, cudaStream_t s) {
+    const unsigned grid = (unsigned)((h->B + 255) / 256);
+    grbs_select_kernel<<<grid, 256, 0, s>>>(h->mask_g, h->mask_r, h->sel_list, h->sel_count + h->flip,
+                                            h->sel_count + (h->flip ^ 1), h->B, h->block_begin,
+                                            (uint32_t)(h->seed & 0xffffffffu), (uint32_t)(h->seed >> 32),
+                                            (uint32_t)(h->t & 0xffffffffu), (uint32_t)(h->t >> 32),
+                                            h->R1, h->R2, is_reset ? 1 : 0, draw ? 1 : 0);
     h->launches++;
     CU_TRY(cudaGetLastError());
+    h->flip ^= 1;   // the counter just filled is sel_count[h->flip ^ 1] from here on
     return CSER_OK;
 }
 
-template <int V, int U>
+template <int V>
 int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t s) {
     const long long cols = P.c_end - P.c_begin;
     if (cols <= 0) return CSER_OK;
-    const long long grid_ll = (cols + 255) / 256;
-    if (grid_ll > 0x7fffffffll) return fail(CSER_ERR_INVALID, "vector too long for one launch");
+    const long long tiles = (cols + kStepThreads - 1) / kStepThreads;
+    const long long grid_ll = tiles * P.n + P.sel_ctas;
+    if (grid_ll > 0x7fffffffll) return fail(CSER_ERR_INVALID, "n_workers * d too large for one launch");
+    StepParams Q = P;
+    Q.tiles = (unsigned)tiles;
     const unsigned grid = (unsigned)grid_ll;
     const bool mom = h->m != nullptr;
     if (mom) {
-        if (is_reset) cser_step_kernel<V, true, true, U><<<grid, 256, 0, s>>>(P);
-        else          cser_step_kernel<V, true, false, U><<<grid, 256, 0, s>>>(P);
+        if (is_reset) cser_step_kernel<V, true, true><<<grid, kStepThreads, 0, s>>>(Q);
+        else          cser_step_kernel<V, true, false><<<grid, kStepThreads, 0, s>>>(Q);
     } else {
-        if (is_reset) cser_step_kernel<V, false, true, U><<<grid, 256, 0, s>>>(P);
-        else          cser_step_kernel<V, false, false, U><<<grid, 256, 0, s>>>(P);
+        if (is_reset) cser_step_kernel<V, false, true><<<grid, kStepThreads, 0, s>>>(Q);
+        else          cser_step_kernel<V, false, false><<<grid, kStepThreads, 0, s>>>(Q);
     }
     h->launches++;
     CU_TRY(cudaGetLastError());
@@ -366,16 +495,20 @@ int launch_step(cser_ctx *h, const float *grad, long long col0, long long col1, 
     StepParams P;
     P.g = grad, P.x = h->x, P.e = h->e, P.m = h->m;
     P.mask_g = h->mask_g, P.mask_r = h->mask_r;
+    P.list = h->sel_list, P.count = h->sel_count + (h->flip ^ 1);
+    P.sel_ctas = (unsigned)h->sel_ctas, P.tiles = 0;
     P.d = h->d, P.n = h->n;
     P.eta = h->eta, P.beta = h->beta, P.n_f = (float)h->n;
     const bool v4 = h->vec4 && ((uintptr_t)grad % 16 == 0) && (col0 % 4 == 0) &&
                     (col1 % 4 == 0 || col1 == h->d);
     if (v4) {
         P.c_begin = col0 / 4, P.c_end = col1 / 4, P.bsv = (unsigned)(h->bs / 4);
-        return launch_step_v<4, 2>(h, P, is_reset, s);
+        P.cols_total = h->d / 4;
+        return launch_step_v<4>(h, P, is_reset, s);
     }
     P.c_begin = col0, P.c_end = col1, P.bsv = (unsigned)h->bs;
-    return launch_step_v<1, 4>(h, P, is_reset, s);
+    P.cols_total = h->d;
+    return launch_step_v<1>(h, P, is_reset, s);
 }
 
 int check_handle(cser_ctx *h) {
@@ -449,6 +582,12 @@ cser_handle cser_create_slab(int64_t d, int32_t n_workers, int32_t block_size, u
     if (er == cudaSuccess) er = cudaMemset(h->x, 0, bytes);
     if (er == cudaSuccess) er = cudaMemset(h->e, 0, bytes);
     if (er == cudaSuccess && h->m) er = cudaMemset(h->m, 0, bytes);
+    if (er == cudaSuccess) er = cudaMalloc(&h->sel_list, (size_t)B * sizeof(uint32_t));
+    if (er == cudaSuccess) er = cudaMalloc(&h->sel_count, 2 * sizeof(uint32_t));
+    if (er == cudaSuccess) er = cudaMemset(h->sel_count, 0, 2 * sizeof(uint32_t));
+    int sms = 0;
+    if (er == cudaSuccess) er = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
+    h->sel_ctas = kSelCtasPerSm * (sms > 0 ? sms : 1);
     if (er == cudaSuccess) er = cudaMemset(h->mask_g, 0, (size_t)B);
     if (er == cudaSuccess) er = cudaMemset(h->mask_r, 0, (size_t)B);
     for (int k = 0; k < 3 && er == cudaSuccess; ++k) er = cudaEventCreate(&h->ev[k]);
@@ -472,6 +611,7 @@ void cser_destroy(cser_handle h) {
     if (!h) return;
     cudaFree(h->x), cudaFree(h->e), cudaFree(h->m);
     cudaFree(h->mask_g), cudaFree(h->mask_r), cudaFree(h->x0_stage), cudaFree(h->g_stage);
+    cudaFree(h->sel_list), cudaFree(h->sel_count);
     for (auto &ev : h->ev) if (ev) cudaEventDestroy(ev);
     for (auto &ev : h->h_ev) if (ev) cudaEventDestroy(ev);
     for (auto &s : h->hs) if (s) cudaStreamDestroy(s);
@@ -507,9 +647,7 @@ int cser_step(cser_handle h, const float *grad, void *stream) {
     cudaStream_t s = (cudaStream_t)stream;
     const bool is_reset = begin_iteration(h);
     if (h->timing) CU_TRY(cudaEventRecord(h->ev[0], s));
-    if (!h->masks_injected) {
-        if (int rc = launch_masks(h, is_reset, s)) return rc;
-    }
+    if (int rc = launch_select(h, is_reset, !h->masks_injected, s)) return rc;
     h->masks_injected = false;
     if (h->timing) CU_TRY(cudaEventRecord(h->ev[1], s));
     if (int rc = launch_step(h, grad, 0, h->d, is_reset, s)) return rc;
@@ -531,9 +669,7 @@ int cser_step_host(cser_handle h, const float *grad_host, void *stream) {
     }
     const bool is_reset = begin_iteration(h);
     // masks first, on the caller's stream; both internal streams start after them
-    if (!h->masks_injected) {
-        if (int rc = launch_masks(h, is_reset, s)) return rc;
-    }
+    if (int rc = launch_select(h, is_reset, !h->masks_injected, s)) return rc;
     h->masks_injected = false;
     CU_TRY(cudaEventRecord(h->h_ev[0], s));
     CU_TRY(cudaStreamWaitEvent(h->hs[0], h->h_ev[0], 0));
@@ -660,19 +796,25 @@ int64_t cser_launch_count(cser_handle h) { return h ? h->launches : 0; }
 }  // extern "C"
 
 // ------------------------------------------------------------------ allocation-free step
-// The two GRBS masks are the only scratch memory a step needs.  For callers that must
-// not allocate, they live here: a fixed array that every GPU which loads this library
-// keeps until the process exits (2 * CSER_NOALLOC_MAX_BLOCKS bytes).  The first half
-// holds the update mask, the second half the reset mask.
-static __device__ __align__(256) uint8_t g_noalloc_masks[2 * CSER_NOALLOC_MAX_BLOCKS];
+// A step's only scratch is what the select kernel hands to the step kernel: the two GRBS
+// masks, the list of selected blocks and two list counters.  For callers that must not
+// allocate, that scratch lives here: a fixed array that every GPU which loads this
+// library keeps until the process exits.  Layout (bytes): update mask [0, MAXB), reset
+// mask [MAXB, 2 MAXB), list of uint32 [2 MAXB, 6 MAXB), two uint32 counters after it.
+// Static device memory starts zeroed, which is the state the counters need.
+constexpr size_t kNoallocMaxB = CSER_NOALLOC_MAX_BLOCKS;
+constexpr size_t kNoallocBytes = 6 * kNoallocMaxB + 256;
+static __device__ __align__(256) uint8_t g_noalloc_scratch[kNoallocBytes];
 
 namespace {
 
 constexpr int kNoallocMaxDevices = 64;
-// Device address of g_noalloc_masks on each device, looked up once per device.  In host
+// Device address of g_noalloc_scratch on each device, looked up once per device.  In host
 // code the array's name is only a handle for the runtime, never an address a kernel may
 // be given; cudaGetSymbolAddress translates it for the device that is current.
 uint8_t *g_noalloc_addr[kNoallocMaxDevices] = {};
+int g_noalloc_flip[kNoallocMaxDevices] = {};      // which counter the next call uses
+int g_noalloc_sel_ctas[kNoallocMaxDevices] = {};
 
 int noalloc_scratch(int device, uint8_t **out) {
     if (device < 0 || device >= kNoallocMaxDevices)
@@ -680,12 +822,20 @@ int noalloc_scratch(int device, uint8_t **out) {
     uint8_t *p = __atomic_load_n(&g_noalloc_addr[device], __ATOMIC_ACQUIRE);
     if (!p) {
         void *sym = nullptr;
-        cudaError_t er = cudaGetSymbolAddress(&sym, g_noalloc_masks);
+        cudaError_t er = cudaGetSymbolAddress(&sym, g_noalloc_scratch);
         if (er != cudaSuccess || !sym) {
             cudaGetLastError();
             return fail(CSER_ERR_CUDA, "cser_step_noalloc: cudaGetSymbolAddress: %s",
                         cudaGetErrorString(er));
         }
+        int sms = 0;
+        er = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+        if (er != cudaSuccess) {
+            cudaGetLastError();
+            return fail(CSER_ERR_CUDA, "cser_step_noalloc: cudaDeviceGetAttribute: %s",
+                        cudaGetErrorString(er));
+        }
+        g_noalloc_sel_ctas[device] = kSelCtasPerSm * (sms > 0 ? sms : 1);
         p = static_cast<uint8_t *>(sym);
         __atomic_store_n(&g_noalloc_addr[device], p, __ATOMIC_RELEASE);
     }
@@ -720,19 +870,26 @@ extern "C" int cser_step_noalloc(int64_t d, int32_t n_workers, int32_t block_siz
 
     cser_ctx c;   // plain stack object describing the caller's arrays; owns nothing
     CU_TRY(cudaGetDevice(&c.device));
-    uint8_t *masks = nullptr;
-    if (int rc = noalloc_scratch(c.device, &masks)) return rc;
+    uint8_t *scratch = nullptr;
+    if (int rc = noalloc_scratch(c.device, &scratch)) return rc;
     c.d = d, c.n = n_workers, c.bs = block_size, c.R1 = R1, c.R2 = R2, c.H = H;
     c.eta = eta, c.beta = beta, c.seed = seed, c.B = B, c.block_begin = 0;
     c.t = t;
     c.x = x, c.e = e, c.m = (beta != 0.f) ? m : nullptr;
-    c.mask_g = masks, c.mask_r = masks + CSER_NOALLOC_MAX_BLOCKS;
+    c.mask_g = scratch, c.mask_r = scratch + kNoallocMaxB;
+    c.sel_list = reinterpret_cast<uint32_t *>(scratch + 2 * kNoallocMaxB);
+    c.sel_count = reinterpret_cast<uint32_t *>(scratch + 6 * kNoallocMaxB);
+    c.flip = g_noalloc_flip[c.device];
+    c.sel_ctas = g_noalloc_sel_ctas[c.device];
     c.vec4 = (d % 4 == 0) && (block_size % 4 == 0) &&
              (((uintptr_t)x | (uintptr_t)e | (uintptr_t)c.m) % 16 == 0);
     const bool is_reset = (t % (uint64_t)H) == 0;
     cudaStream_t s = (cudaStream_t)stream;
-    // Both masks are rewritten for all B blocks before the step kernel reads them, so
-    // nothing left in the array by an earlier call is ever used.
-    if (int rc = launch_masks(&c, is_reset, s)) return rc;
+    // The select kernel rewrites every mask entry and list entry the step kernel reads and
+    // clears the counter the next call will use, so nothing an earlier call left in the
+    // array is ever used and nothing has to be cleared between calls.
+    const int rc = launch_select(&c, is_reset, true, s);
+    g_noalloc_flip[c.device] = c.flip;
+    if (rc) return rc;
     return launch_step(&c, grad, 0, d, is_reset, s);
 }
