@@ -3,14 +3,14 @@
 //
 // Layout: g, x, e, m are fp32 [n, d] row-major (worker-major).  The step is bound
 // by HBM traffic (about 28 bytes per element and worker against 7 flops), so the
-// kernel is organised around how DRAM likes to be walked: the grid is (column
-// tiles, workers) and CTAs are dispatched tile-fastest, so the unselected blocks
+// step is organised around how DRAM likes to be walked: the streaming kernel's grid
+// is (workers x column tiles), dispatched tile-fastest, so the unselected blocks
 // (all but 1/R of the data, purely elementwise) are streamed row after row as four
 // long contiguous read streams and three write streams, every byte touched once.
-// Blocks selected by a mask (1/R of the data) need the mean over workers: an extra
-// row of CTAs, dispatched first, handles them with 8 worker lanes per column that
-// meet in shared memory.  There is no contraction here and tensor cores are not
-// used.
+// Blocks selected by a mask (1/R of the data) need the mean over workers: the
+// select kernel compacts their ids into a list and a second kernel, with its own
+// register budget, walks the worker axis for exactly those columns.  There is no
+// contraction here and tensor cores are not used.
 //
 // Compiled with -fmad=false: every multiply and add rounds separately, in the
 // order stated in include/cser.h.
@@ -173,7 +173,6 @@ struct StepParams {
     long long c_end;         // one past the last
     unsigned bsv;            // GRBS block size in vector columns
     unsigned tiles;          // tiles of 256 vector columns in [c_begin, c_end)
-    unsigned sel_ctas;       // leading CTAs of the grid that work on the selected blocks
     int n;
     float eta, beta, n_f;
 };
@@ -196,197 +195,179 @@ __device__ __forceinline__ Pack<V> get_p(const Pack<V> &g, Pack<V> &m, float eta
     return p;
 }
 
-// Shape of the CTA that handles selected columns: 32 vector columns x 8 worker lanes.
-constexpr int kSelCols = 32;
-constexpr int kSelLanes = 8;
-constexpr int kStepThreads = kSelCols * kSelLanes;   // 256
-#ifndef CSER_SEL_CTAS_PER_SM
-#define CSER_SEL_CTAS_PER_SM 4
-#endif
-constexpr int kSelCtasPerSm = CSER_SEL_CTAS_PER_SM;  // CTAs per SM given to the selected blocks
+constexpr int kStepThreads = 256;   // streaming kernel: one CTA = 256 vector columns of one row
+constexpr int kWalkThreads = 128;   // selected-block kernel
+constexpr int kWalkBatch = 4;       // workers whose loads a walking thread keeps in flight
 
-// Ordered sum over the workers of one lane chunk: acc = ((acc + S[0]) + S[1]) + ...,
-// starting from S[0] itself when `first` (no 0.0f is ever added).
-template <int V>
-__device__ __forceinline__ void ordered_accumulate(Pack<V> &acc, const Pack<V> (*S)[kSelCols], int cv,
-                                                   int cnt, bool first) {
-    for (int k = 0; k < cnt; ++k) {
-        const Pack<V> s = S[k][cv];
-#pragma unroll
-        for (int q = 0; q < V; ++q) acc.v[q] = (first && k == 0) ? s.v[q] : acc.v[q] + s.v[q];
-    }
-}
-
-// Selected blocks, all workers.  The first P.sel_ctas CTAs of the grid share the list of
-// selected blocks in pieces of at most 256 vector columns.  A piece is walked in chunks of
-// 32 columns; in a chunk, warp w owns worker lane w, so every access is one contiguous run
-// of a row, and the workers' values of a column meet in shared memory, where they are
-// summed in ascending worker order.  A block's two mask flags are uniform over the CTA.
+// Selected blocks (1/R of the data): the update needs the mean over workers, so here one
+// thread owns one vector column of a selected block and walks the worker axis.  Threads
+// are laid over the concatenation of the listed blocks, so CTAs are full whatever the
+// block size.  Each pass issues the loads of kWalkBatch workers before it consumes any of
+// them (the in-place stores would otherwise keep the compiler from hoisting the next
+// worker's loads), and sums in ascending worker order starting from worker 0's value.
+// This kernel has its own register budget; the streaming kernel stays at 32 registers.
 template <int V, bool MOM, bool RESET>
-__device__ __forceinline__ void selected_blocks_role(const StepParams &P) {
-    __shared__ Pack<V> S[2][kSelLanes][kSelCols];
-    const int cv = threadIdx.x & (kSelCols - 1);
-    const int wl = threadIdx.x / kSelCols;
+__global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepParams P) {
+    constexpr int U = kWalkBatch;
+    const unsigned long long total = (unsigned long long)(*P.count) * P.bsv;
     const long long d = P.d;
     const int n = P.n;
     const float eta = P.eta, beta = P.beta;
-    const unsigned pieces_per_block = (P.bsv + kStepThreads - 1) / kStepThreads;
-    const unsigned long long items = (unsigned long long)(*P.count) * pieces_per_block;
-    int buf = 0;
-
-    for (unsigned long long w = blockIdx.x; w < items; w += P.sel_ctas) {
-        const unsigned blk = P.list[w / pieces_per_block];
-        const unsigned piece = (unsigned)(w % pieces_per_block);
+    for (unsigned long long f = (unsigned long long)blockIdx.x * kWalkThreads + threadIdx.x; f < total;
+         f += (unsigned long long)gridDim.x * kWalkThreads) {
+        const unsigned long long entry = (total <= 0xffffffffull) ? (unsigned long long)((uint32_t)f / P.bsv)
+                                                                  : f / P.bsv;
+        const unsigned blk = P.list[entry];
+        const long long c = (long long)blk * P.bsv + (long long)(f - entry * P.bsv);
+        if (c >= P.cols_total || c < P.c_begin || c >= P.c_end) continue;
         const bool sg = P.mask_g[blk] != 0;
         const bool sr = RESET ? (P.mask_r[blk] != 0) : false;
-        const bool only_r = sr && !sg;
-        const long long blk_c0 = (long long)blk * P.bsv;
-        long long c_lo = blk_c0 + (long long)piece * kStepThreads;
-        long long c_hi = min(min(c_lo + kStepThreads, blk_c0 + (long long)P.bsv), P.cols_total);
-        c_lo = max(c_lo, P.c_begin);
-        c_hi = min(c_hi, P.c_end);
+        const float *__restrict__ g = P.g + c * V;
+        float *__restrict__ x = P.x + c * V;
+        float *__restrict__ e = P.e + c * V;
+        float *__restrict__ m = MOM ? P.m + c * V : nullptr;
+        Pack<V> sum_e;   // sum over workers of e_{t-1/2} (reset-selected blocks)
+#pragma unroll
+        for (int k = 0; k < V; ++k) sum_e.v[k] = 0.f;
 
-        for (long long cc = c_lo; cc < c_hi; cc += kSelCols) {
-            const long long c = cc + cv;
-            const bool valid = c < c_hi;
-            const float *__restrict__ g = P.g + c * V;
-            float *__restrict__ x = P.x + c * V;
-            float *__restrict__ e = P.e + c * V;
-            float *__restrict__ m = MOM ? P.m + c * V : nullptr;
-            Pack<V> sum_p, sum_e;
+        if (sg) {
+            // Update-selected block: r = 0, p' = mean_k p_k.  Pass A forms the mean and updates m.
+            Pack<V> sum_p;
 #pragma unroll
-            for (int q = 0; q < V; ++q) sum_p.v[q] = sum_e.v[q] = 0.f;
-
-            // The first round's x (and e) of an update-selected block are fetched together
-            // with its g and m, so that a chunk costs one memory round trip, not two.
-            Pack<V> x0v, e0v;
+            for (int k = 0; k < V; ++k) sum_p.v[k] = 0.f;
+            for (int i0 = 0; i0 < n; i0 += U) {
+                Pack<V> gv[U], mv[U];
 #pragma unroll
-            for (int q = 0; q < V; ++q) x0v.v[q] = e0v.v[q] = 0.f;
-            if (sg && valid && wl < n) {
-                x0v = ld<V>(x + (long long)wl * d);
-                if (sr) e0v = ld<V>(e + (long long)wl * d);
-            }
-
-            // Pass 1: Get_p for every worker.  An update-selected block gathers sum_k p_k.
-            // A block selected by the reset mask only takes its own residual step here
-            // (x_{t-1/2} = x - p, e_{t-1/2} = e - p), stores x_{t-1/2} - e_{t-1/2}, zeroes
-            // e and gathers sum_k e_{k,t-1/2}.
-            for (int i0 = 0; i0 < n; i0 += kSelLanes) {
-                const int i = i0 + wl;
-                const long long o = (long long)i * d;
-                Pack<V> p, eh;
-#pragma unroll
-                for (int q = 0; q < V; ++q) p.v[q] = eh.v[q] = 0.f;
-                if (valid && i < n) {
-                    const Pack<V> gv = ld_stream<V>(g + o);
-                    Pack<V> mv, xv, ev;
-                    if constexpr (MOM) mv = ld<V>(m + o);
-                    if (only_r) {
-                        xv = ld<V>(x + o);
-                        ev = ld<V>(e + o);
-                    }
-                    p = get_p<V, MOM>(gv, mv, eta, beta);
-                    if constexpr (MOM) st<V>(m + o, mv);
-                    if (only_r) {
-                        Pack<V> z;
-#pragma unroll
-                        for (int q = 0; q < V; ++q) {
-                            const float xh = xv.v[q] - p.v[q];
-                            eh.v[q] = ev.v[q] - p.v[q];
-                            xv.v[q] = xh - eh.v[q];
-                            z.v[q] = 0.f;
-                        }
-                        st<V>(x + o, xv);
-                        st<V>(e + o, z);
+                for (int u = 0; u < U; ++u) {
+                    if (i0 + u < n) {
+                        const long long o = (long long)(i0 + u) * d;
+                        gv[u] = ld_stream<V>(g + o);
+                        if constexpr (MOM) mv[u] = ld<V>(m + o);
                     }
                 }
-                S[buf][wl][cv] = only_r ? eh : p;
-                __syncthreads();
-                ordered_accumulate<V>(only_r ? sum_e : sum_p, S[buf], cv, min(kSelLanes, n - i0), i0 == 0);
-                buf ^= 1;                                // the next round writes the other buffer
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    if (i0 + u < n) {
+                        const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], eta, beta);
+                        if constexpr (MOM) st<V>(m + (long long)(i0 + u) * d, mv[u]);
+#pragma unroll
+                        for (int k = 0; k < V; ++k)
+                            sum_p.v[k] = (i0 + u == 0) ? p.v[k] : sum_p.v[k] + p.v[k];
+                    }
+                }
             }
-
-            // Pass 2 (update-selected block): x_i -= mean_k p_k; e untouched.  If the block is
-            // reset-selected too: store (x_i - p-bar) - e_i, zero e, gather sum_k e_k.
-            if (sg) {
-                Pack<V> pbar;
+            Pack<V> pbar;
 #pragma unroll
-                for (int q = 0; q < V; ++q) pbar.v[q] = sum_p.v[q] / P.n_f;
-                for (int i0 = 0; i0 < n; i0 += kSelLanes) {
-                    const int i = i0 + wl;
-                    const long long o = (long long)i * d;
-                    Pack<V> ev;
+            for (int k = 0; k < V; ++k) pbar.v[k] = sum_p.v[k] / P.n_f;
+            // Pass B: x_i -= p-bar; e untouched.  If the block is reset-selected too: store
+            // (x_i - p-bar) - e_i, zero e, gather sum_k e_k.
+            for (int i0 = 0; i0 < n; i0 += U) {
+                Pack<V> xv[U], ev[U];
 #pragma unroll
-                    for (int q = 0; q < V; ++q) ev.v[q] = 0.f;
-                    if (valid && i < n) {
-                        Pack<V> xv = x0v;
-                        if (i0 == 0) {
-                            ev = e0v;
-                        } else {
-                            xv = ld<V>(x + o);
-                            if (sr) ev = ld<V>(e + o);
-                        }
+                for (int u = 0; u < U; ++u) {
+                    if (i0 + u < n) {
+                        const long long o = (long long)(i0 + u) * d;
+                        xv[u] = ld<V>(x + o);
+                        if (sr) ev[u] = ld<V>(e + o);
+                    }
+                }
 #pragma unroll
-                        for (int q = 0; q < V; ++q) xv.v[q] = xv.v[q] - pbar.v[q];
+                for (int u = 0; u < U; ++u) {
+                    if (i0 + u < n) {
+                        const long long o = (long long)(i0 + u) * d;
+#pragma unroll
+                        for (int k = 0; k < V; ++k) xv[u].v[k] = xv[u].v[k] - pbar.v[k];
                         if (sr) {
                             Pack<V> z;
 #pragma unroll
-                            for (int q = 0; q < V; ++q) {
-                                xv.v[q] = xv.v[q] - ev.v[q];
-                                z.v[q] = 0.f;
+                            for (int k = 0; k < V; ++k) {
+                                sum_e.v[k] = (i0 + u == 0) ? ev[u].v[k] : sum_e.v[k] + ev[u].v[k];
+                                xv[u].v[k] = xv[u].v[k] - ev[u].v[k];
+                                z.v[k] = 0.f;
                             }
                             st<V>(e + o, z);
                         }
-                        st<V>(x + o, xv);
-                    }
-                    if (sr) {
-                        S[buf][wl][cv] = ev;
-                        __syncthreads();
-                        ordered_accumulate<V>(sum_e, S[buf], cv, min(kSelLanes, n - i0), i0 == 0);
-                        buf ^= 1;
+                        st<V>(x + o, xv[u]);
                     }
                 }
             }
+        } else {
+            // Selected by the reset mask only: take the residual step (x_{t-1/2} = x - p,
+            // e_{t-1/2} = e - p), store x_{t-1/2} - e_{t-1/2}, zero e, gather sum_k e_{k,t-1/2}.
+            constexpr int U2 = 2;
+            for (int i0 = 0; i0 < n; i0 += U2) {
+                Pack<V> gv[U2], mv[U2], xv[U2], ev[U2];
+#pragma unroll
+                for (int u = 0; u < U2; ++u) {
+                    if (i0 + u < n) {
+                        const long long o = (long long)(i0 + u) * d;
+                        gv[u] = ld_stream<V>(g + o);
+                        if constexpr (MOM) mv[u] = ld<V>(m + o);
+                        xv[u] = ld<V>(x + o);
+                        ev[u] = ld<V>(e + o);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U2; ++u) {
+                    if (i0 + u < n) {
+                        const long long o = (long long)(i0 + u) * d;
+                        const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], eta, beta);
+                        if constexpr (MOM) st<V>(m + o, mv[u]);
+                        Pack<V> z;
+#pragma unroll
+                        for (int k = 0; k < V; ++k) {
+                            const float xh = xv[u].v[k] - p.v[k];
+                            const float eh = ev[u].v[k] - p.v[k];
+                            sum_e.v[k] = (i0 + u == 0) ? eh : sum_e.v[k] + eh;
+                            xv[u].v[k] = xh - eh;
+                            z.v[k] = 0.f;
+                        }
+                        st<V>(x + o, xv[u]);
+                        st<V>(e + o, z);
+                    }
+                }
+            }
+        }
 
-            // Pass 3 (reset-selected block), Algorithm 2 lines 11-12:
+        if (sr) {
+            // Error reset (Algorithm 2 lines 11-12):
             // x_i = (x_{i,t-1/2} - e_{i,t-1/2}) + mean_k e_{k,t-1/2}.
-            if (sr && valid) {
-                Pack<V> ebar;
+            Pack<V> ebar;
 #pragma unroll
-                for (int q = 0; q < V; ++q) ebar.v[q] = sum_e.v[q] / P.n_f;
-                for (int i = wl; i < n; i += kSelLanes) {
-                    const long long o = (long long)i * d;
-                    Pack<V> xv = ld<V>(x + o);
+            for (int k = 0; k < V; ++k) ebar.v[k] = sum_e.v[k] / P.n_f;
+            for (int i0 = 0; i0 < n; i0 += U) {
+                Pack<V> xv[U];
 #pragma unroll
-                    for (int q = 0; q < V; ++q) xv.v[q] = xv.v[q] + ebar.v[q];
-                    st<V>(x + o, xv);
+                for (int u = 0; u < U; ++u)
+                    if (i0 + u < n) xv[u] = ld<V>(x + (long long)(i0 + u) * d);
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    if (i0 + u < n) {
+#pragma unroll
+                        for (int k = 0; k < V; ++k) xv[u].v[k] = xv[u].v[k] + ebar.v[k];
+                        st<V>(x + (long long)(i0 + u) * d, xv[u]);
+                    }
                 }
             }
         }
     }
 }
 
-// 1-D grid.  CTAs [0, sel_ctas), dispatched first, work on the selected blocks.  CTA
-// sel_ctas + i * tiles + tile streams tile `tile` of worker i: thread t owns vector column
-// c = c_begin + 256 * tile + t and updates it element by element unless a mask selects
-// its block.  Consecutive CTAs walk one row after the other, contiguously.
+// Unselected blocks (all but 1/R of the data), purely elementwise.  1-D grid: CTA
+// i * tiles + tile streams tile `tile` of worker i, so consecutive CTAs walk one row after
+// the other, contiguously.  Thread t owns vector column c = c_begin + 256 * tile + t and
+// leaves it alone if a mask selects its block.
 template <int V, bool MOM, bool RESET>
-__global__ void __launch_bounds__(kStepThreads, 8) cser_step_kernel(const StepParams P) {
-    if (blockIdx.x < P.sel_ctas) {
-        selected_blocks_role<V, MOM, RESET>(P);
-        return;
-    }
-    const unsigned id = blockIdx.x - P.sel_ctas;
-    const unsigned row = id / P.tiles;
-    const unsigned tile = id - row * P.tiles;
+__global__ void __launch_bounds__(kStepThreads, 8) cser_stream_kernel(const StepParams P) {
+    const unsigned row = blockIdx.x / P.tiles;
+    const unsigned tile = blockIdx.x - row * P.tiles;
     const long long c = P.c_begin + (long long)tile * kStepThreads + threadIdx.x;
     if (c >= P.c_end) return;
     const long long b = (P.c_end <= 0xffffffffll) ? (long long)((uint32_t)c / P.bsv)
                                                   : (long long)((unsigned long long)c / P.bsv);
     if (P.mask_g[b] != 0) return;
     if (RESET && P.mask_r[b] != 0) return;
-    // Unselected block, no reset: C(p) = 0, so p' = r = p (Algorithm 3 lines 4-8):
-    // x_i -= p_i, e_i -= p_i.  Purely elementwise.
+    // C(p) = 0, so p' = r = p (Algorithm 3 lines 4-8): x_i -= p_i, e_i -= p_i.
     const long long o = (long long)row * P.d + c * V;
     const Pack<V> gv = ld_stream<V>(P.g + o);
     Pack<V> mv;
@@ -433,7 +414,11 @@ struct cser_ctx {
     uint32_t *sel_list = nullptr;                    // [B] blocks selected this step
     uint32_t *sel_count = nullptr;                   // [2] counters, used alternately
     int flip = 0;                                    // which counter the next step uses
-    int sel_ctas = 0;                                // CTAs of the step kernel given to selected blocks
+    bool walk_all = false;                           // masks were injected: no estimate of the selected count
+    // The selected-block kernel and the streaming kernel touch disjoint columns; with an
+    // auxiliary stream they run side by side (fork after the select kernel, join after both).
+    cudaStream_t aux = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     float *x0_stage = nullptr;                       // [d] staging for a host x0
     bool masks_injected = false;
     bool vec4 = false;                               // 128-bit path usable for the state arrays
@@ -467,36 +452,65 @@ int launch_select(cser_ctx *h, bool is_reset, bool draw, cudaStream_t s) {
 }
 
 template <int V>
-int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t s) {
+int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t s, bool use_aux) {
     const long long cols = P.c_end - P.c_begin;
     if (cols <= 0) return CSER_OK;
     const long long tiles = (cols + kStepThreads - 1) / kStepThreads;
-    const long long grid_ll = tiles * P.n + P.sel_ctas;
+    const long long grid_ll = tiles * P.n;
     if (grid_ll > 0x7fffffffll) return fail(CSER_ERR_INVALID, "n_workers * d too large for one launch");
     StepParams Q = P;
     Q.tiles = (unsigned)tiles;
     const unsigned grid = (unsigned)grid_ll;
+    // Grid of the selected-block kernel: the count lives on the device, so size the grid for
+    // the expected number of selected columns in this launch's range plus slack; the kernel
+    // strides over whatever the list really holds, so any grid size is correct.
+    double frac = h->walk_all ? 1.0 : 1.0 / h->R1 + (is_reset ? 1.0 / h->R2 : 0.0);
+    if (frac > 1.0) frac = 1.0;
+    const double exp_blocks = frac * ((double)cols / P.bsv + 1.0);
+    const double blocks = exp_blocks + 6.0 * sqrt(exp_blocks) + 4.0;
+    long long wgrid = (long long)(blocks * P.bsv / kWalkThreads) + 1;
+    const long long wmax = (cols + kWalkThreads - 1) / kWalkThreads + 1;
+    if (wgrid > wmax) wgrid = wmax;
     const bool mom = h->m != nullptr;
-    if (mom) {
-        if (is_reset) cser_step_kernel<V, true, true><<<grid, kStepThreads, 0, s>>>(Q);
-        else          cser_step_kernel<V, true, false><<<grid, kStepThreads, 0, s>>>(Q);
-    } else {
-        if (is_reset) cser_step_kernel<V, false, true><<<grid, kStepThreads, 0, s>>>(Q);
-        else          cser_step_kernel<V, false, false><<<grid, kStepThreads, 0, s>>>(Q);
+    // R1 == 1 selects every block on every step: nothing is left to stream.
+    const bool stream_any = h->walk_all || h->R1 != 1;
+    cudaStream_t ws = s;
+    const bool fork = use_aux && h->aux != nullptr && stream_any;
+    if (fork) {
+        CU_TRY(cudaEventRecord(h->ev_fork, s));
+        CU_TRY(cudaStreamWaitEvent(h->aux, h->ev_fork, 0));
+        ws = h->aux;
     }
-    h->launches++;
+#define CSER_LAUNCH_PAIR(MOM_, RESET_)                                                                  \
+    do {                                                                                                \
+        cser_selected_kernel<V, MOM_, RESET_><<<(unsigned)wgrid, kWalkThreads, 0, ws>>>(Q);             \
+        if (stream_any) cser_stream_kernel<V, MOM_, RESET_><<<grid, kStepThreads, 0, s>>>(Q);           \
+    } while (0)
+    if (mom) {
+        if (is_reset) CSER_LAUNCH_PAIR(true, true);
+        else          CSER_LAUNCH_PAIR(true, false);
+    } else {
+        if (is_reset) CSER_LAUNCH_PAIR(false, true);
+        else          CSER_LAUNCH_PAIR(false, false);
+    }
+#undef CSER_LAUNCH_PAIR
+    h->launches += stream_any ? 2 : 1;
     CU_TRY(cudaGetLastError());
+    if (fork) {
+        CU_TRY(cudaEventRecord(h->ev_join, h->aux));
+        CU_TRY(cudaStreamWaitEvent(s, h->ev_join, 0));
+    }
     return CSER_OK;
 }
 
 // Launch the fused step kernel on element columns [col0, col1) of gradients `grad`.
 int launch_step(cser_ctx *h, const float *grad, long long col0, long long col1, bool is_reset,
-                cudaStream_t s) {
+                cudaStream_t s, bool use_aux = false) {
     StepParams P;
     P.g = grad, P.x = h->x, P.e = h->e, P.m = h->m;
     P.mask_g = h->mask_g, P.mask_r = h->mask_r;
     P.list = h->sel_list, P.count = h->sel_count + (h->flip ^ 1);
-    P.sel_ctas = (unsigned)h->sel_ctas, P.tiles = 0;
+    P.tiles = 0;
     P.d = h->d, P.n = h->n;
     P.eta = h->eta, P.beta = h->beta, P.n_f = (float)h->n;
     const bool v4 = h->vec4 && ((uintptr_t)grad % 16 == 0) && (col0 % 4 == 0) &&
@@ -504,11 +518,11 @@ int launch_step(cser_ctx *h, const float *grad, long long col0, long long col1, 
     if (v4) {
         P.c_begin = col0 / 4, P.c_end = col1 / 4, P.bsv = (unsigned)(h->bs / 4);
         P.cols_total = h->d / 4;
-        return launch_step_v<4>(h, P, is_reset, s);
+        return launch_step_v<4>(h, P, is_reset, s, use_aux);
     }
     P.c_begin = col0, P.c_end = col1, P.bsv = (unsigned)h->bs;
     P.cols_total = h->d;
-    return launch_step_v<1>(h, P, is_reset, s);
+    return launch_step_v<1>(h, P, is_reset, s, use_aux);
 }
 
 int check_handle(cser_ctx *h) {
@@ -585,12 +599,16 @@ cser_handle cser_create_slab(int64_t d, int32_t n_workers, int32_t block_size, u
     if (er == cudaSuccess) er = cudaMalloc(&h->sel_list, (size_t)B * sizeof(uint32_t));
     if (er == cudaSuccess) er = cudaMalloc(&h->sel_count, 2 * sizeof(uint32_t));
     if (er == cudaSuccess) er = cudaMemset(h->sel_count, 0, 2 * sizeof(uint32_t));
-    int sms = 0;
-    if (er == cudaSuccess) er = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device);
-    h->sel_ctas = kSelCtasPerSm * (sms > 0 ? sms : 1);
     if (er == cudaSuccess) er = cudaMemset(h->mask_g, 0, (size_t)B);
     if (er == cudaSuccess) er = cudaMemset(h->mask_r, 0, (size_t)B);
     for (int k = 0; k < 3 && er == cudaSuccess; ++k) er = cudaEventCreate(&h->ev[k]);
+    if (er == cudaSuccess) {
+        int lo = 0, hi = 0;   // hi = numerically lowest = highest priority
+        er = cudaDeviceGetStreamPriorityRange(&lo, &hi);
+        if (er == cudaSuccess) er = cudaStreamCreateWithPriority(&h->aux, cudaStreamNonBlocking, hi);
+    }
+    if (er == cudaSuccess) er = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
+    if (er == cudaSuccess) er = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
     if (er == cudaSuccess) er = cudaDeviceSynchronize();
     if (er != cudaSuccess) {
         fail(er == cudaErrorMemoryAllocation ? CSER_ERR_NOMEM : CSER_ERR_CUDA, "cser_create: %s",
@@ -615,6 +633,9 @@ void cser_destroy(cser_handle h) {
     for (auto &ev : h->ev) if (ev) cudaEventDestroy(ev);
     for (auto &ev : h->h_ev) if (ev) cudaEventDestroy(ev);
     for (auto &s : h->hs) if (s) cudaStreamDestroy(s);
+    if (h->aux) cudaStreamDestroy(h->aux);
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_join) cudaEventDestroy(h->ev_join);
     delete h;
 }
 
@@ -648,9 +669,10 @@ int cser_step(cser_handle h, const float *grad, void *stream) {
     const bool is_reset = begin_iteration(h);
     if (h->timing) CU_TRY(cudaEventRecord(h->ev[0], s));
     if (int rc = launch_select(h, is_reset, !h->masks_injected, s)) return rc;
+    h->walk_all = h->masks_injected;
     h->masks_injected = false;
     if (h->timing) CU_TRY(cudaEventRecord(h->ev[1], s));
-    if (int rc = launch_step(h, grad, 0, h->d, is_reset, s)) return rc;
+    if (int rc = launch_step(h, grad, 0, h->d, is_reset, s, true)) return rc;
     if (h->timing) {
         CU_TRY(cudaEventRecord(h->ev[2], s));
         h->ev_valid = true;
@@ -670,6 +692,7 @@ int cser_step_host(cser_handle h, const float *grad_host, void *stream) {
     const bool is_reset = begin_iteration(h);
     // masks first, on the caller's stream; both internal streams start after them
     if (int rc = launch_select(h, is_reset, !h->masks_injected, s)) return rc;
+    h->walk_all = h->masks_injected;
     h->masks_injected = false;
     CU_TRY(cudaEventRecord(h->h_ev[0], s));
     CU_TRY(cudaStreamWaitEvent(h->hs[0], h->h_ev[0], 0));
@@ -814,7 +837,6 @@ constexpr int kNoallocMaxDevices = 64;
 // be given; cudaGetSymbolAddress translates it for the device that is current.
 uint8_t *g_noalloc_addr[kNoallocMaxDevices] = {};
 int g_noalloc_flip[kNoallocMaxDevices] = {};      // which counter the next call uses
-int g_noalloc_sel_ctas[kNoallocMaxDevices] = {};
 
 int noalloc_scratch(int device, uint8_t **out) {
     if (device < 0 || device >= kNoallocMaxDevices)
@@ -828,14 +850,6 @@ int noalloc_scratch(int device, uint8_t **out) {
             return fail(CSER_ERR_CUDA, "cser_step_noalloc: cudaGetSymbolAddress: %s",
                         cudaGetErrorString(er));
         }
-        int sms = 0;
-        er = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
-        if (er != cudaSuccess) {
-            cudaGetLastError();
-            return fail(CSER_ERR_CUDA, "cser_step_noalloc: cudaDeviceGetAttribute: %s",
-                        cudaGetErrorString(er));
-        }
-        g_noalloc_sel_ctas[device] = kSelCtasPerSm * (sms > 0 ? sms : 1);
         p = static_cast<uint8_t *>(sym);
         __atomic_store_n(&g_noalloc_addr[device], p, __ATOMIC_RELEASE);
     }
@@ -880,7 +894,6 @@ extern "C" int cser_step_noalloc(int64_t d, int32_t n_workers, int32_t block_siz
     c.sel_list = reinterpret_cast<uint32_t *>(scratch + 2 * kNoallocMaxB);
     c.sel_count = reinterpret_cast<uint32_t *>(scratch + 6 * kNoallocMaxB);
     c.flip = g_noalloc_flip[c.device];
-    c.sel_ctas = g_noalloc_sel_ctas[c.device];
     c.vec4 = (d % 4 == 0) && (block_size % 4 == 0) &&
              (((uintptr_t)x | (uintptr_t)e | (uintptr_t)c.m) % 16 == 0);
     const bool is_reset = (t % (uint64_t)H) == 0;
