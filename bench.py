@@ -24,10 +24,11 @@ METRIC = "cser_steps_per_sec"
 UNIT = "steps/s"
 PEAK_NOMINAL_GBS = 8000.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused step kernel.  Captured with
-# ncu on the same workload cut to d = 8,388,608 (1.8074e9 bytes per launch) and scaled by d, traffic
-# being proportional to d; see profiles/cser_step_kernel_cfg2_d8M_ncu_full.md.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2_wrn40x8_n8_R32_H8": 1.8074e9 * 35_748_708 / 8_388_608}
+# dram__bytes_read.sum + dram__bytes_write.sum per step of the streaming kernel plus the selected-block
+# kernel.  Captured with ncu on the same workload cut to d = 8,388,608 (1.7658e9 + 0.0325e9 bytes per
+# step) and scaled by d, traffic being proportional to d; see
+# profiles/cser_stream_and_selected_kernels_cfg2_d8M_ncu_full.md.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2_wrn40x8_n8_R32_H8": 1.7983e9 * 35_748_708 / 8_388_608}
 
 
 def algorithmic_bytes(w, frac_e_touched):
