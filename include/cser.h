@@ -78,7 +78,10 @@ typedef struct cser_ctx *cser_handle;
  *   d           > 0, elements per worker
  *   n_workers   > 0
  *   block_size  > 0, elements per GRBS block (last block may be short)
- *   R1, R2      >= 1, compression ratios of the update / reset compressors
+ *   R1          compression ratio of the update compressor; R1 = 1 keeps everything,
+ *               R1 = 0 keeps nothing (C = 0: the special cases CSER-PL and, with H = 1,
+ *               CSEA of Appendix A.1, where nothing is exchanged between resets)
+ *   R2          >= 1, compression ratio of the reset compressor
  *   H           > 0, error-reset interval
  *   eta         finite learning rate;  beta in [0, 1): 0 = no momentum (m is not
  *               allocated, read or written)
@@ -100,6 +103,21 @@ cser_handle cser_create(int64_t d, int32_t n_workers, int32_t block_size,
 cser_handle cser_create_slab(int64_t d, int32_t n_workers, int32_t block_size,
                              uint32_t R1, uint32_t R2, int32_t H,
                              float eta, float beta, uint64_t seed, int64_t block_begin);
+
+/*
+ * General form.  flags:
+ *   CSER_FLAG_NO_ERROR_ARRAY  "implementation II" of Appendix A.4: with GRBS a block's
+ *       residual is either already part of the local model or reset to zero, so no error
+ *       array is kept; on a reset step the reset-selected blocks of x are replaced by
+ *       their mean over workers (PSync applied to x itself).  State is x (and m) only;
+ *       CSER_STATE_E cannot be read or written.  The models equal implementation I's up
+ *       to rounding.
+ */
+#define CSER_FLAG_NO_ERROR_ARRAY 1u
+cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size,
+                           uint32_t R1, uint32_t R2, int32_t H,
+                           float eta, float beta, uint64_t seed, int64_t block_begin,
+                           uint32_t flags);
 
 /* Free everything the handle owns.  The caller must have synchronized its streams. NULL is ignored. */
 void cser_destroy(cser_handle h);
@@ -152,7 +170,7 @@ int cser_debug_set_masks(cser_handle h, const uint8_t *g_mask, const uint8_t *r_
 /*
  * Stand-alone GRBS block-select kernel (Definition 2): writes uint8 flags of blocks
  * block_begin .. block_begin + n_blocks - 1 at step t for compressor `which`
- * (0 = update, 1 = reset) with ratio R into device memory `mask_out`.
+ * (0 = update, 1 = reset) with ratio R (0 = nothing selected) into device memory `mask_out`.
  */
 int cser_grbs_mask(uint64_t seed, uint64_t t, uint32_t which, int64_t block_begin,
                    int64_t n_blocks, uint32_t R, uint8_t *mask_out, void *stream);

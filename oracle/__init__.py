@@ -6,7 +6,7 @@ This package is a plain, slow restatement of the paper's algorithms in NumPy:
 * ``grbs``    - the globally-randomized blockwise sparsifier mask (Definition 2)
 * ``cser``    - PSync (Algorithm 3), Get_p (Appendix A.4), CSER (Algorithm 2),
                 M-CSER implementation I (Algorithm 4) and the memory-saving
-                implementation II (Appendix A.4)
+                implementation II (Appendix A.4) and the special case CSEA (Appendix A.1)
 
 It exists only so that tests, the smoke check and the benchmark's CPU-baseline
 leg can compare the CUDA library against something that can be checked against
@@ -18,4 +18,4 @@ exact rational brute force, library generators); none is "parity unpinned".
 """
 from .philox import philox4x32_10, philox4_generic          # noqa: F401
 from .grbs import grbs_mask, n_blocks, STREAM_GRAD, STREAM_RESET   # noqa: F401
-from .cser import psync, get_p, CSEROracle, CSERImpl2Oracle  # noqa: F401
+from .cser import psync, get_p, CSEROracle, CSERImpl2Oracle, CSEAOracle  # noqa: F401

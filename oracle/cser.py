@@ -9,6 +9,7 @@ intermediate vectors v', r and v-bar':
 * ``get_p``            - Appendix A.4, "Calculate update on worker i"
 * ``CSEROracle``       - Algorithm 2 (beta = 0) and Algorithm 4 (beta != 0)
 * ``CSERImpl2Oracle``  - Appendix A.4, implementation II (no error array)
+* ``CSEAOracle``       - Appendix A.1, CSEA (implementation I), the special case C2 = 0, H = 1
 
 Arithmetic runs in ``dtype``: float64 (default) is the reference trajectory;
 float32 evaluates the same expressions in the storage precision, one IEEE
@@ -153,3 +154,26 @@ class CSERImpl2Oracle(_Base):
         self.x = self.x - p_prime
         if is_reset:
             self.x, _ = psync(self.x, sel_r)
+
+
+class CSEAOracle(_Base):
+    """Appendix A.1, "CSEA (Implementation I)": SGD with error assimilation, the special case
+    of CSER with C2 = 0 and H = 1, in the paper's own three-line form (no momentum):
+        p_i  <- e_i - eta * g_i
+        e'_i, e_i <- PSync(p_i, C1)
+        x_i  <- x_i + e'_i - e_{i,t-1}
+    The last line is applied to the whole vector, as printed."""
+
+    def __init__(self, d, n_workers, block_size, R2, eta, seed, dtype=np.float64, cols=None):
+        super().__init__(d, n_workers, block_size, 0, R2, 1, eta, 0.0, seed, dtype=dtype, cols=cols)
+        self.e = np.zeros_like(self.x)
+
+    def step(self, g):
+        g = np.asarray(g, self.dtype)
+        self.t += 1
+        self.mask_r = grbs_mask(self.seed, self.t, STREAM_RESET, self.B, self.R2)
+        sel = self.mask_r[self.block_of_col] != 0
+        e_old = self.e
+        p = e_old - self.eta * g
+        e_prime, self.e = psync(p, sel)
+        self.x = self.x + e_prime - e_old

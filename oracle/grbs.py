@@ -11,7 +11,9 @@ expectation exactly as Definition 2 states.
 Draw: word 0 of Philox4x32-10 with key = (seed low 32 bits, seed high 32 bits)
 and counter = (b, t low 32 bits, t high 32 bits, stream), stream 0 for the
 per-step compressor of the update, 1 for the error-reset compressor.  Block b
-is selected iff  word0 * R < 2**32  (R = 1 selects everything).
+is selected iff  word0 * R < 2**32  (R = 1 selects everything).  R = 0 stands for the
+compressor C = 0 that keeps nothing (delta = 0, allowed by Definition 1 as extended in
+Section 3): the special cases CSER-PL and CSEA of Appendix A.1.
 """
 import numpy as np
 from .philox import philox4x32_10
@@ -26,6 +28,8 @@ def n_blocks(d, block_size):
 
 def grbs_mask(seed, t, stream, B, R, block_begin=0):
     """uint8[B] selection flags of blocks block_begin .. block_begin+B-1 at step t."""
+    if int(R) == 0:
+        return np.zeros(B, np.uint8)
     seed = int(seed) & 0xFFFFFFFFFFFFFFFF
     t = int(t) & 0xFFFFFFFFFFFFFFFF
     b = np.arange(block_begin, block_begin + B, dtype=np.uint64)

@@ -37,6 +37,8 @@ def lib():
                               c.c_float, c.c_float, c.c_uint64]
     L.cser_create_slab.restype = c.c_void_p
     L.cser_create_slab.argtypes = L.cser_create.argtypes + [c.c_int64]
+    L.cser_create_ex.restype = c.c_void_p
+    L.cser_create_ex.argtypes = L.cser_create_slab.argtypes + [c.c_uint32]
     L.cser_destroy.restype = None
     L.cser_destroy.argtypes = [c.c_void_p]
     L.cser_set_x0.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p]
@@ -81,8 +83,11 @@ def _ptr(t):
     return ctypes.c_void_p(t.data_ptr())
 
 
-def cser_create(d, n_workers, block_size, R1, R2, H, eta, beta, seed, block_begin=0):
-    h = lib().cser_create_slab(d, n_workers, block_size, R1, R2, H, eta, beta, seed, block_begin)
+FLAG_NO_ERROR_ARRAY = 1
+
+
+def cser_create(d, n_workers, block_size, R1, R2, H, eta, beta, seed, block_begin=0, flags=0):
+    h = lib().cser_create_ex(d, n_workers, block_size, R1, R2, H, eta, beta, seed, block_begin, flags)
     if not h:
         raise CSERError(f"cser_create failed: {cser_last_error()}")
     return ctypes.c_void_p(h)
@@ -152,10 +157,10 @@ def cser_launch_count(h):
 class CSER:
     """Convenience owner of one handle (still only marshalling)."""
 
-    def __init__(self, d, n_workers, block_size, R1, R2, H, eta, beta, seed=0, block_begin=0):
+    def __init__(self, d, n_workers, block_size, R1, R2, H, eta, beta, seed=0, block_begin=0, flags=0):
         self.d, self.n, self.bs, self.beta = int(d), int(n_workers), int(block_size), float(beta)
         self.B = (self.d + self.bs - 1) // self.bs
-        self.h = cser_create(d, n_workers, block_size, R1, R2, H, eta, beta, seed, block_begin)
+        self.h = cser_create(d, n_workers, block_size, R1, R2, H, eta, beta, seed, block_begin, flags)
 
     def close(self):
         if self.h is not None:

@@ -78,7 +78,7 @@ grbs_mask_kernel(uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r, lon
     const uint32_t R = which ? R_r : R_g;
     const uint32_t w0 =
         philox4x32_10_word0(k0, k1, (uint32_t)(block_begin + b), t_lo, t_hi, which);
-    const uint8_t sel = ((unsigned long long)w0 * R < (1ull << 32)) ? 1 : 0;
+    const uint8_t sel = (R != 0 && (unsigned long long)w0 * R < (1ull << 32)) ? 1 : 0;   // R = 0: C = 0
     (second ? mask_r : mask_g)[b] = sel;
 }
 
@@ -99,7 +99,8 @@ grbs_select_kernel(uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r,
     if (b < B) {
         if (draw) {
             const uint32_t gb = (uint32_t)(block_begin + b);
-            sg = (unsigned long long)philox4x32_10_word0(k0, k1, gb, t_lo, t_hi, 0u) * R_g < (1ull << 32);
+            sg = R_g != 0 &&   // R1 = 0: the update compressor keeps nothing (C = 0)
+                 (unsigned long long)philox4x32_10_word0(k0, k1, gb, t_lo, t_hi, 0u) * R_g < (1ull << 32);
             mask_g[b] = sg ? 1 : 0;
             if (is_reset) {
                 sr = (unsigned long long)philox4x32_10_word0(k0, k1, gb, t_lo, t_hi, 1u) * R_r < (1ull << 32);
@@ -206,7 +207,7 @@ constexpr int kWalkBatch = 4;       // workers whose loads a walking thread keep
 // them (the in-place stores would otherwise keep the compiler from hoisting the next
 // worker's loads), and sums in ascending worker order starting from worker 0's value.
 // This kernel has its own register budget; the streaming kernel stays at 32 registers.
-template <int V, bool MOM, bool RESET>
+template <int V, bool MOM, bool RESET, bool ERR>
 __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepParams P) {
     constexpr int U = kWalkBatch;
     const unsigned long long total = (unsigned long long)(*P.count) * P.bsv;
@@ -224,11 +225,13 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
         const bool sr = RESET ? (P.mask_r[blk] != 0) : false;
         const float *__restrict__ g = P.g + c * V;
         float *__restrict__ x = P.x + c * V;
-        float *__restrict__ e = P.e + c * V;
+        float *__restrict__ e = ERR ? P.e + c * V : nullptr;
         float *__restrict__ m = MOM ? P.m + c * V : nullptr;
-        Pack<V> sum_e;   // sum over workers of e_{t-1/2} (reset-selected blocks)
+        // With an error array: sum over workers of e_{t-1/2}.  Without one (implementation
+        // II): sum over workers of x_{t-1/2}.  Reset-selected blocks only.
+        Pack<V> sum_r;
 #pragma unroll
-        for (int k = 0; k < V; ++k) sum_e.v[k] = 0.f;
+        for (int k = 0; k < V; ++k) sum_r.v[k] = 0.f;
 
         if (sg) {
             // Update-selected block: r = 0, p' = mean_k p_k.  Pass A forms the mean and updates m.
@@ -259,8 +262,9 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
             Pack<V> pbar;
 #pragma unroll
             for (int k = 0; k < V; ++k) pbar.v[k] = sum_p.v[k] / P.n_f;
-            // Pass B: x_i -= p-bar; e untouched.  If the block is reset-selected too: store
-            // (x_i - p-bar) - e_i, zero e, gather sum_k e_k.
+            // Pass B: x_i -= p-bar; e untouched.  If the block is reset-selected too: with an
+            // error array store (x_i - p-bar) - e_i, zero e and gather sum_k e_k; without one
+            // gather sum_k (x_k - p-bar) and store nothing yet.
             for (int i0 = 0; i0 < n; i0 += U) {
                 Pack<V> xv[U], ev[U];
 #pragma unroll
@@ -268,7 +272,9 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
                     if (i0 + u < n) {
                         const long long o = (long long)(i0 + u) * d;
                         xv[u] = ld<V>(x + o);
-                        if (sr) ev[u] = ld<V>(e + o);
+                        if constexpr (ERR) {
+                            if (sr) ev[u] = ld<V>(e + o);
+                        }
                     }
                 }
 #pragma unroll
@@ -278,22 +284,31 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
 #pragma unroll
                         for (int k = 0; k < V; ++k) xv[u].v[k] = xv[u].v[k] - pbar.v[k];
                         if (sr) {
-                            Pack<V> z;
+                            if constexpr (ERR) {
+                                Pack<V> z;
 #pragma unroll
-                            for (int k = 0; k < V; ++k) {
-                                sum_e.v[k] = (i0 + u == 0) ? ev[u].v[k] : sum_e.v[k] + ev[u].v[k];
-                                xv[u].v[k] = xv[u].v[k] - ev[u].v[k];
-                                z.v[k] = 0.f;
+                                for (int k = 0; k < V; ++k) {
+                                    sum_r.v[k] = (i0 + u == 0) ? ev[u].v[k] : sum_r.v[k] + ev[u].v[k];
+                                    xv[u].v[k] = xv[u].v[k] - ev[u].v[k];
+                                    z.v[k] = 0.f;
+                                }
+                                st<V>(e + o, z);
+                                st<V>(x + o, xv[u]);
+                            } else {
+#pragma unroll
+                                for (int k = 0; k < V; ++k)
+                                    sum_r.v[k] = (i0 + u == 0) ? xv[u].v[k] : sum_r.v[k] + xv[u].v[k];
                             }
-                            st<V>(e + o, z);
+                        } else {
+                            st<V>(x + o, xv[u]);
                         }
-                        st<V>(x + o, xv[u]);
                     }
                 }
             }
         } else {
             // Selected by the reset mask only: take the residual step (x_{t-1/2} = x - p,
-            // e_{t-1/2} = e - p), store x_{t-1/2} - e_{t-1/2}, zero e, gather sum_k e_{k,t-1/2}.
+            // e_{t-1/2} = e - p).  With an error array store x_{t-1/2} - e_{t-1/2}, zero e and
+            // gather sum_k e_{k,t-1/2}; without one gather sum_k x_{k,t-1/2}.
             constexpr int U2 = 2;
             for (int i0 = 0; i0 < n; i0 += U2) {
                 Pack<V> gv[U2], mv[U2], xv[U2], ev[U2];
@@ -304,7 +319,7 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
                         gv[u] = ld_stream<V>(g + o);
                         if constexpr (MOM) mv[u] = ld<V>(m + o);
                         xv[u] = ld<V>(x + o);
-                        ev[u] = ld<V>(e + o);
+                        if constexpr (ERR) ev[u] = ld<V>(e + o);
                     }
                 }
 #pragma unroll
@@ -313,41 +328,54 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
                         const long long o = (long long)(i0 + u) * d;
                         const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], eta, beta);
                         if constexpr (MOM) st<V>(m + o, mv[u]);
-                        Pack<V> z;
+                        if constexpr (ERR) {
+                            Pack<V> z;
 #pragma unroll
-                        for (int k = 0; k < V; ++k) {
-                            const float xh = xv[u].v[k] - p.v[k];
-                            const float eh = ev[u].v[k] - p.v[k];
-                            sum_e.v[k] = (i0 + u == 0) ? eh : sum_e.v[k] + eh;
-                            xv[u].v[k] = xh - eh;
-                            z.v[k] = 0.f;
+                            for (int k = 0; k < V; ++k) {
+                                const float xh = xv[u].v[k] - p.v[k];
+                                const float eh = ev[u].v[k] - p.v[k];
+                                sum_r.v[k] = (i0 + u == 0) ? eh : sum_r.v[k] + eh;
+                                xv[u].v[k] = xh - eh;
+                                z.v[k] = 0.f;
+                            }
+                            st<V>(x + o, xv[u]);
+                            st<V>(e + o, z);
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < V; ++k) {
+                                const float xh = xv[u].v[k] - p.v[k];
+                                sum_r.v[k] = (i0 + u == 0) ? xh : sum_r.v[k] + xh;
+                            }
                         }
-                        st<V>(x + o, xv[u]);
-                        st<V>(e + o, z);
                     }
                 }
             }
         }
 
         if (sr) {
-            // Error reset (Algorithm 2 lines 11-12):
-            // x_i = (x_{i,t-1/2} - e_{i,t-1/2}) + mean_k e_{k,t-1/2}.
-            Pack<V> ebar;
+            Pack<V> rbar;
 #pragma unroll
-            for (int k = 0; k < V; ++k) ebar.v[k] = sum_e.v[k] / P.n_f;
-            for (int i0 = 0; i0 < n; i0 += U) {
-                Pack<V> xv[U];
+            for (int k = 0; k < V; ++k) rbar.v[k] = sum_r.v[k] / P.n_f;
+            if constexpr (ERR) {
+                // Error reset (Algorithm 2 lines 11-12):
+                // x_i = (x_{i,t-1/2} - e_{i,t-1/2}) + mean_k e_{k,t-1/2}.
+                for (int i0 = 0; i0 < n; i0 += U) {
+                    Pack<V> xv[U];
 #pragma unroll
-                for (int u = 0; u < U; ++u)
-                    if (i0 + u < n) xv[u] = ld<V>(x + (long long)(i0 + u) * d);
+                    for (int u = 0; u < U; ++u)
+                        if (i0 + u < n) xv[u] = ld<V>(x + (long long)(i0 + u) * d);
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    if (i0 + u < n) {
+                    for (int u = 0; u < U; ++u) {
+                        if (i0 + u < n) {
 #pragma unroll
-                        for (int k = 0; k < V; ++k) xv[u].v[k] = xv[u].v[k] + ebar.v[k];
-                        st<V>(x + (long long)(i0 + u) * d, xv[u]);
+                            for (int k = 0; k < V; ++k) xv[u].v[k] = xv[u].v[k] + rbar.v[k];
+                            st<V>(x + (long long)(i0 + u) * d, xv[u]);
+                        }
                     }
                 }
+            } else {
+                // Implementation II (Appendix A.4): x_i = mean_k x_{k,t-1/2} for every worker.
+                for (int i = 0; i < n; ++i) st<V>(x + (long long)i * d, rbar);
             }
         }
     }
@@ -357,7 +385,7 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
 // i * tiles + tile streams tile `tile` of worker i, so consecutive CTAs walk one row after
 // the other, contiguously.  Thread t owns vector column c = c_begin + 256 * tile + t and
 // leaves it alone if a mask selects its block.
-template <int V, bool MOM, bool RESET>
+template <int V, bool MOM, bool RESET, bool ERR>
 __global__ void __launch_bounds__(kStepThreads, 8) cser_stream_kernel(const StepParams P) {
     const unsigned row = blockIdx.x / P.tiles;
     const unsigned tile = blockIdx.x - row * P.tiles;
@@ -367,22 +395,24 @@ __global__ void __launch_bounds__(kStepThreads, 8) cser_stream_kernel(const Step
                                                   : (long long)((unsigned long long)c / P.bsv);
     if (P.mask_g[b] != 0) return;
     if (RESET && P.mask_r[b] != 0) return;
-    // C(p) = 0, so p' = r = p (Algorithm 3 lines 4-8): x_i -= p_i, e_i -= p_i.
+    // C(p) = 0, so p' = r = p (Algorithm 3 lines 4-8): x_i -= p_i, e_i -= p_i (no e array in
+    // implementation II).
     const long long o = (long long)row * P.d + c * V;
     const Pack<V> gv = ld_stream<V>(P.g + o);
     Pack<V> mv;
     if constexpr (MOM) mv = ld<V>(P.m + o);
     Pack<V> xv = ld<V>(P.x + o);
-    Pack<V> ev = ld<V>(P.e + o);
+    Pack<V> ev;
+    if constexpr (ERR) ev = ld<V>(P.e + o);
     const Pack<V> p = get_p<V, MOM>(gv, mv, P.eta, P.beta);
 #pragma unroll
     for (int k = 0; k < V; ++k) {
         xv.v[k] = xv.v[k] - p.v[k];
-        ev.v[k] = ev.v[k] - p.v[k];
+        if constexpr (ERR) ev.v[k] = ev.v[k] - p.v[k];
     }
     if constexpr (MOM) st<V>(P.m + o, mv);
     st<V>(P.x + o, xv);
-    st<V>(P.e + o, ev);
+    if constexpr (ERR) st<V>(P.e + o, ev);
 }
 
 // x_i <- x0 for all workers; e, m <- 0
@@ -395,7 +425,7 @@ broadcast_x0_kernel(const float *__restrict__ x0, float *__restrict__ x, float *
     for (int i = 0; i < n; ++i) {
         const long long o = (long long)i * d + j;
         x[o] = v;
-        e[o] = 0.f;
+        if (e) e[o] = 0.f;
         if (m) m[o] = 0.f;
     }
 }
@@ -464,7 +494,7 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     // Grid of the selected-block kernel: the count lives on the device, so size the grid for
     // the expected number of selected columns in this launch's range plus slack; the kernel
     // strides over whatever the list really holds, so any grid size is correct.
-    double frac = h->walk_all ? 1.0 : 1.0 / h->R1 + (is_reset ? 1.0 / h->R2 : 0.0);
+    double frac = h->walk_all ? 1.0 : (h->R1 ? 1.0 / h->R1 : 0.0) + (is_reset ? 1.0 / h->R2 : 0.0);
     if (frac > 1.0) frac = 1.0;
     const double exp_blocks = frac * ((double)cols / P.bsv + 1.0);
     const double blocks = exp_blocks + 6.0 * sqrt(exp_blocks) + 4.0;
@@ -481,18 +511,25 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
         CU_TRY(cudaStreamWaitEvent(h->aux, h->ev_fork, 0));
         ws = h->aux;
     }
-#define CSER_LAUNCH_PAIR(MOM_, RESET_)                                                                  \
+    const bool err = h->e != nullptr;
+#define CSER_LAUNCH_PAIR(MOM_, RESET_, ERR_)                                                            \
     do {                                                                                                \
-        cser_selected_kernel<V, MOM_, RESET_><<<(unsigned)wgrid, kWalkThreads, 0, ws>>>(Q);             \
-        if (stream_any) cser_stream_kernel<V, MOM_, RESET_><<<grid, kStepThreads, 0, s>>>(Q);           \
+        cser_selected_kernel<V, MOM_, RESET_, ERR_><<<(unsigned)wgrid, kWalkThreads, 0, ws>>>(Q);       \
+        if (stream_any) cser_stream_kernel<V, MOM_, RESET_, ERR_><<<grid, kStepThreads, 0, s>>>(Q);     \
+    } while (0)
+#define CSER_LAUNCH_ERR(MOM_, RESET_)                                                                   \
+    do {                                                                                                \
+        if (err) CSER_LAUNCH_PAIR(MOM_, RESET_, true);                                                  \
+        else     CSER_LAUNCH_PAIR(MOM_, RESET_, false);                                                 \
     } while (0)
     if (mom) {
-        if (is_reset) CSER_LAUNCH_PAIR(true, true);
-        else          CSER_LAUNCH_PAIR(true, false);
+        if (is_reset) CSER_LAUNCH_ERR(true, true);
+        else          CSER_LAUNCH_ERR(true, false);
     } else {
-        if (is_reset) CSER_LAUNCH_PAIR(false, true);
-        else          CSER_LAUNCH_PAIR(false, false);
+        if (is_reset) CSER_LAUNCH_ERR(false, true);
+        else          CSER_LAUNCH_ERR(false, false);
     }
+#undef CSER_LAUNCH_ERR
 #undef CSER_LAUNCH_PAIR
     h->launches += stream_any ? 2 : 1;
     CU_TRY(cudaGetLastError());
@@ -560,13 +597,16 @@ extern "C" {
 
 const char *cser_last_error(void) { return g_err; }
 
-cser_handle cser_create_slab(int64_t d, int32_t n_workers, int32_t block_size, uint32_t R1,
-                             uint32_t R2, int32_t H, float eta, float beta, uint64_t seed,
-                             int64_t block_begin) {
+cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uint32_t R1,
+                           uint32_t R2, int32_t H, float eta, float beta, uint64_t seed,
+                           int64_t block_begin, uint32_t flags) {
     g_err[0] = 0;
-    if (d <= 0 || n_workers <= 0 || block_size <= 0 || R1 == 0 || R2 == 0 || H <= 0 ||
-        block_begin < 0) {
-        fail(CSER_ERR_INVALID, "cser_create: d, n_workers, block_size, R1, R2, H must be positive");
+    if (d <= 0 || n_workers <= 0 || block_size <= 0 || R2 == 0 || H <= 0 || block_begin < 0) {
+        fail(CSER_ERR_INVALID, "cser_create: d, n_workers, block_size, R2, H must be positive");
+        return nullptr;
+    }
+    if (flags & ~(uint32_t)CSER_FLAG_NO_ERROR_ARRAY) {
+        fail(CSER_ERR_INVALID, "cser_create: unknown flags 0x%x", flags);
         return nullptr;
     }
     if (!isfinite(eta) || !(beta >= 0.f && beta < 1.f)) {
@@ -589,12 +629,13 @@ cser_handle cser_create_slab(int64_t d, int32_t n_workers, int32_t block_size, u
     const size_t bytes = state_elems(h) * sizeof(float);
     cudaError_t er = cudaGetDevice(&h->device);
     if (er == cudaSuccess) er = cudaMalloc(&h->x, bytes);
-    if (er == cudaSuccess) er = cudaMalloc(&h->e, bytes);
+    const bool with_e = !(flags & CSER_FLAG_NO_ERROR_ARRAY);
+    if (er == cudaSuccess && with_e) er = cudaMalloc(&h->e, bytes);
     if (er == cudaSuccess && beta != 0.f) er = cudaMalloc(&h->m, bytes);
     if (er == cudaSuccess) er = cudaMalloc(&h->mask_g, (size_t)B);
     if (er == cudaSuccess) er = cudaMalloc(&h->mask_r, (size_t)B);
     if (er == cudaSuccess) er = cudaMemset(h->x, 0, bytes);
-    if (er == cudaSuccess) er = cudaMemset(h->e, 0, bytes);
+    if (er == cudaSuccess && h->e) er = cudaMemset(h->e, 0, bytes);
     if (er == cudaSuccess && h->m) er = cudaMemset(h->m, 0, bytes);
     if (er == cudaSuccess) er = cudaMalloc(&h->sel_list, (size_t)B * sizeof(uint32_t));
     if (er == cudaSuccess) er = cudaMalloc(&h->sel_count, 2 * sizeof(uint32_t));
@@ -620,9 +661,15 @@ cser_handle cser_create_slab(int64_t d, int32_t n_workers, int32_t block_size, u
     return h;
 }
 
+cser_handle cser_create_slab(int64_t d, int32_t n_workers, int32_t block_size, uint32_t R1,
+                             uint32_t R2, int32_t H, float eta, float beta, uint64_t seed,
+                             int64_t block_begin) {
+    return cser_create_ex(d, n_workers, block_size, R1, R2, H, eta, beta, seed, block_begin, 0);
+}
+
 cser_handle cser_create(int64_t d, int32_t n_workers, int32_t block_size, uint32_t R1, uint32_t R2,
                         int32_t H, float eta, float beta, uint64_t seed) {
-    return cser_create_slab(d, n_workers, block_size, R1, R2, H, eta, beta, seed, 0);
+    return cser_create_ex(d, n_workers, block_size, R1, R2, H, eta, beta, seed, 0, 0);
 }
 
 void cser_destroy(cser_handle h) {
@@ -722,7 +769,10 @@ int cser_step_host(cser_handle h, const float *grad_host, void *stream) {
 static int state_piece(cser_ctx *h, int which, void **ptr, size_t *bytes) {
     switch (which) {
         case CSER_STATE_X: *ptr = h->x, *bytes = state_elems(h) * sizeof(float); return CSER_OK;
-        case CSER_STATE_E: *ptr = h->e, *bytes = state_elems(h) * sizeof(float); return CSER_OK;
+        case CSER_STATE_E:
+            if (!h->e) return fail(CSER_ERR_INVALID, "no error array (CSER_FLAG_NO_ERROR_ARRAY)");
+            *ptr = h->e, *bytes = state_elems(h) * sizeof(float);
+            return CSER_OK;
         case CSER_STATE_M:
             if (!h->m) return fail(CSER_ERR_INVALID, "no momentum state (beta == 0)");
             *ptr = h->m, *bytes = state_elems(h) * sizeof(float);
@@ -863,9 +913,9 @@ extern "C" int cser_step_noalloc(int64_t d, int32_t n_workers, int32_t block_siz
                                  uint32_t R2, int32_t H, float eta, float beta, uint64_t seed,
                                  uint64_t t, const float *grad, float *x, float *e, float *m,
                                  void *stream) {
-    if (d <= 0 || n_workers <= 0 || block_size <= 0 || R1 == 0 || R2 == 0 || H <= 0 || t == 0)
+    if (d <= 0 || n_workers <= 0 || block_size <= 0 || R2 == 0 || H <= 0 || t == 0)
         return fail(CSER_ERR_INVALID,
-                    "cser_step_noalloc: d, n_workers, block_size, R1, R2, H, t must be positive");
+                    "cser_step_noalloc: d, n_workers, block_size, R2, H, t must be positive");
     if (!isfinite(eta) || !(beta >= 0.f && beta < 1.f))
         return fail(CSER_ERR_INVALID, "cser_step_noalloc: eta must be finite and beta in [0, 1)");
     const long long B = (d + block_size - 1) / block_size;

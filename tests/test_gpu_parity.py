@@ -14,7 +14,7 @@ import pytest
 import torch
 
 from _golden import read_hand_example
-from oracle import CSEROracle, grbs_mask, n_blocks, philox4x32_10, STREAM_GRAD, STREAM_RESET
+from oracle import CSEAOracle, CSERImpl2Oracle, CSEROracle, grbs_mask, n_blocks, philox4x32_10, STREAM_GRAD, STREAM_RESET
 from paper_2007_13221_b200 import binding as b, synth
 
 pytestmark = pytest.mark.gpu
@@ -80,11 +80,12 @@ def test_oracle_philox_matches_curand_library():
 
 
 # ------------------------------------------------------------------ small shapes, element by element
-def _run_both(d, n, bs, R1, R2, H, eta, beta, steps, seed=3, masks=None, x0=None, grads=None, dtype=np.float32):
+def _run_both(d, n, bs, R1, R2, H, eta, beta, steps, seed=3, masks=None, x0=None, grads=None, dtype=np.float32,
+              flags=0, oracle=CSEROracle):
     rng = np.random.default_rng(1000 + d + n)
     x0 = rng.standard_normal(d).astype(np.float32) if x0 is None else x0
-    opt = b.CSER(d, n, bs, R1, R2, H, eta, beta, seed)
-    ref = CSEROracle(d, n, bs, R1, R2, H, eta, beta, seed, dtype=dtype)
+    opt = b.CSER(d, n, bs, R1, R2, H, eta, beta, seed, flags=flags)
+    ref = oracle(d, n, bs, R1, R2, H, eta, beta, seed, dtype=dtype)
     opt.set_x0(torch.from_numpy(x0).to(DEV))
     ref.set_x0(x0)
     for t in range(1, steps + 1):
@@ -198,8 +199,9 @@ def _cols_of(blocks, w):
     return np.concatenate(parts)
 
 
-def _full_size_parity(cfg, steps=None, n_random=192):
+def _full_size_parity(cfg, steps=None, n_random=192, impl2=False):
     w = synth.CONFIGS[cfg]
+    oracle = CSERImpl2Oracle if impl2 else CSEROracle
     steps = w.steps if steps is None else steps
     rng = np.random.default_rng(cfg)
     B = w.n_blocks
@@ -208,9 +210,10 @@ def _full_size_parity(cfg, steps=None, n_random=192):
     blocks = _sample_blocks(w, masks_g[::max(1, steps // 8)], masks_r[::max(1, len(masks_r) // 8)], rng, n_random)
     cols = _cols_of(blocks, w)
     cols_dev = torch.from_numpy(cols).to(DEV)
-    refs = {dt: CSEROracle(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
-                           dtype=dt, cols=cols) for dt in (np.float32, np.float64)}
-    opt = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed)
+    refs = {dt: oracle(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
+                       dtype=dt, cols=cols) for dt in (np.float32, np.float64)}
+    opt = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
+                 flags=b.FLAG_NO_ERROR_ARRAY if impl2 else 0)
     x0 = synth.x0(w, DEV)
     opt.set_x0(x0)
     x0_s = x0[cols_dev].cpu().numpy()
@@ -218,7 +221,7 @@ def _full_size_parity(cfg, steps=None, n_random=192):
         r.set_x0(x0_s)
     g = torch.empty((w.n_workers, w.d), dtype=torch.float32, device=DEV)
     buf = torch.empty((w.n_workers, w.d), dtype=torch.float32, device=DEV)
-    names = ((b.STATE_X, "x"), (b.STATE_E, "e")) + (((b.STATE_M, "m"),) if w.beta else ())
+    names = ((b.STATE_X, "x"),) + (() if impl2 else ((b.STATE_E, "e"),)) + (((b.STATE_M, "m"),) if w.beta else ())
 
     def compare(rtol, atol_abs, atol_rms):
         for which, name in names:
@@ -241,6 +244,17 @@ def _full_size_parity(cfg, steps=None, n_random=192):
         if t in (1, w.H, steps):
             assert np.array_equal(opt.state(b.STATE_MASK_G).cpu().numpy(), masks_g[t - 1]), t
     compare(1e-4, 0.0, 1e-4)
+    if impl2:
+        # implementation II: right after a reset the reset-selected blocks agree across workers exactly
+        if steps % w.H == 0:
+            b.cser_read_state(opt.h, b.STATE_X, buf)
+            mr = torch.from_numpy(masks_r[-1]).to(DEV).bool()
+            sel_cols = mr.repeat_interleave(w.block_size)[: w.d]
+            assert (buf[:, sel_cols] - buf[0:1, sel_cols]).abs().max().item() == 0.0
+        opt.close()
+        del g, buf
+        torch.cuda.empty_cache()
+        return
     # properties that hold at any size, on the whole state: Lemma 1 and zero error after reset
     b.cser_read_state(opt.h, b.STATE_X, buf)
     b.cser_read_state(opt.h, b.STATE_E, g)
@@ -296,6 +310,65 @@ def test_config5_bert_large_sized_on_sampled_blocks():
     if free < 70 * 2**30:
         pytest.skip("needs about 65 GB of free device memory")
     _full_size_parity(5, n_random=96)
+
+
+# ------------------------------------------------------------------ special cases and implementation II
+@pytest.mark.parametrize("d,n,bs,R2,H,beta", [(4096 + 40, 8, 256, 4, 1, 0.0), (4096 + 40, 8, 256, 2, 4, 0.9),
+                                              (1001, 3, 7, 2, 2, 0.9), (20_000, 16, 1024, 1, 3, 0.0)])
+def test_no_update_sync_special_cases_csea_and_cser_pl(d, n, bs, R2, H, beta):
+    """R1 = 0 (C2 = 0): CSEA when H = 1, CSER-PL otherwise (Appendix A.1)."""
+    opt, ref = _run_both(d, n, bs, 0, R2, H, 0.1, beta, steps=13)
+    for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e")) + (((b.STATE_M, "m"),) if beta else ()):
+        assert np.array_equal(opt.state(which).cpu().numpy(), getattr(ref, name)), name
+    assert not opt.state(b.STATE_MASK_G).any()
+    if H == 1 and beta == 0.0:                      # the paper's own three-line CSEA form
+        rng = np.random.default_rng(1000 + d + n)
+        x0 = rng.standard_normal(d).astype(np.float32)
+        csea = CSEAOracle(d, n, bs, R2, 0.1, 3)
+        csea.set_x0(x0)
+        for _ in range(13):
+            csea.step((rng.standard_normal(d)[None, :] + 0.5 * rng.standard_normal((n, d))).astype(np.float32))
+        got = opt.state(b.STATE_X).cpu().numpy()
+        assert _within(got, csea.x, 1e-5, 1e-5).all()
+    opt.close()
+
+
+@pytest.mark.parametrize("d,n,bs,R1,R2,H,beta", SHAPES)
+def test_implementation_II_equals_its_float32_oracle_exactly(d, n, bs, R1, R2, H, beta):
+    opt, ref = _run_both(d, n, bs, R1, R2, H, 0.1, beta, steps=13, flags=b.FLAG_NO_ERROR_ARRAY,
+                         oracle=CSERImpl2Oracle)
+    for which, name in ((b.STATE_X, "x"),) + (((b.STATE_M, "m"),) if beta else ()):
+        got, want = opt.state(which).cpu().numpy(), getattr(ref, name)
+        bad = got != want
+        assert not bad.any(), (name, int(bad.sum()), np.argwhere(bad)[:5])
+    with pytest.raises(b.CSERError):
+        opt.state(b.STATE_E)
+    opt.close()
+
+
+def test_implementation_II_models_match_implementation_I():
+    d, n, bs = 50_000 + 12, 8, 256
+    a, ra = _run_both(d, n, bs, 4, 2, 4, 0.1, 0.9, steps=40)
+    c, rc = _run_both(d, n, bs, 4, 2, 4, 0.1, 0.9, steps=40, flags=b.FLAG_NO_ERROR_ARRAY, oracle=CSERImpl2Oracle)
+    xa, xc = a.state(b.STATE_X), c.state(b.STATE_X)
+    assert (xa - xc).abs().max().item() <= 1e-4 * xa.abs().max().item()
+    assert torch.equal(a.state(b.STATE_M), c.state(b.STATE_M))
+    a.close(), c.close()
+
+
+def test_all_four_mask_combinations_implementation_II():
+    for d, bs in ((64, 16), (62, 15)):
+        B = n_blocks(d, bs)
+        masks = [([0, 1, 0, 1, 1][:B], [0, 0, 1, 1, 0][:B])] * 3
+        opt, ref = _run_both(d, 4, bs, 2, 2, 1, 0.1, 0.9, steps=3, masks=masks, flags=b.FLAG_NO_ERROR_ARRAY,
+                             oracle=CSERImpl2Oracle)
+        for which, name in ((b.STATE_X, "x"), (b.STATE_M, "m")):
+            assert np.array_equal(opt.state(which).cpu().numpy(), getattr(ref, name)), (d, name)
+        opt.close()
+
+
+def test_implementation_II_full_size_headline_workload_on_sampled_blocks():
+    _full_size_parity(2, impl2=True)
 
 
 # ------------------------------------------------------------------ boundary behaviour
@@ -369,7 +442,8 @@ def test_errors_are_reported_not_raised_on_the_device():
     L = b.lib()
     assert not L.cser_create(0, 8, 256, 4, 4, 4, 0.1, 0.0, 0)
     assert "positive" in b.cser_last_error()
-    assert not L.cser_create(100, 8, 256, 0, 4, 4, 0.1, 0.0, 0)
+    assert not L.cser_create(100, 8, 256, 4, 0, 4, 0.1, 0.0, 0)          # R2 = 0: delta_1 must be positive
+    assert not L.cser_create_ex(100, 8, 256, 4, 4, 4, 0.1, 0.0, 0, 0, 0x80)  # unknown flag
     assert not L.cser_create(100, 8, 256, 4, 4, 0, 0.1, 0.0, 0)
     assert not L.cser_create(100, 8, 256, 4, 4, 4, float("nan"), 0.0, 0)
     assert not L.cser_create(100, 8, 256, 4, 4, 4, 0.1, 1.0, 0)

@@ -14,7 +14,7 @@ import pytest
 
 from _golden import read_hand_example
 
-from oracle import (CSEROracle, CSERImpl2Oracle, grbs_mask, n_blocks, philox4_generic,
+from oracle import (CSEAOracle, CSEROracle, CSERImpl2Oracle, grbs_mask, n_blocks, philox4_generic,
                     philox4x32_10, psync, STREAM_GRAD, STREAM_RESET)
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -393,3 +393,35 @@ def test_float32_evaluation_stays_within_the_stated_tolerances_of_float64():
         rms = np.sqrt((v**2).mean())
         assert (np.abs(u - v) <= 1e-4 * np.abs(v) + 1e-4 * rms).all()
         assert np.abs(u - v).max() <= 1e-5 * np.abs(v).max()
+
+
+# --------------------------------------------------------------------------- C2 = 0 special cases (Appendix A.1)
+def test_ratio_zero_means_the_compressor_keeps_nothing():
+    assert not grbs_mask(3, 5, STREAM_GRAD, 1000, 0).any()
+
+
+def test_csea_is_cser_with_no_update_sync_and_reset_every_step():
+    n, d, T = 4, 600, 20
+    x0, g = _rand_problem(30, n, d, T)
+    a = _run(CSEROracle, g, x0, bs=8, R1=0, R2=4, H=1, eta=0.1, beta=0.0, seed=13)
+    c = CSEAOracle(d, n, 8, 4, 0.1, 13)
+    c.set_x0(x0)
+    for gt in g:
+        c.step(gt)
+        assert not c.e[:, c.mask_r[c.block_of_col] != 0].any()
+    assert np.allclose(a.x, c.x, rtol=1e-12, atol=1e-12) and np.allclose(a.e, c.e, rtol=1e-12, atol=1e-12)
+    assert np.abs(a.x - a.x[0]).max() > 1e-3            # local models do bifurcate
+
+
+def test_cser_pl_with_identity_reset_compressor_is_local_sgd():
+    """C2 = 0 drawn natively (R1 = 0) and delta_1 = 1 (R2 = 1): local SGD with period H."""
+    n, d, T, H, eta = 4, 64, 12, 4, 0.1
+    x0, g = _rand_problem(31, n, d, T)
+    o = _run(CSEROracle, g, x0, bs=8, R1=0, R2=1, H=H, eta=eta, beta=0.0)
+    x = np.repeat(x0.astype(np.float64)[None, :], n, 0)
+    for t, gt in enumerate(g, 1):
+        x = x - float(np.float32(eta)) * gt.astype(np.float64)
+        if t % H == 0:
+            x[:] = x.mean(0)
+    assert np.allclose(o.x, x, rtol=1e-12, atol=1e-12)
+    assert not o.mask_g.any()
