@@ -31,16 +31,21 @@ PEAK_NOMINAL_GBS = 8000.0
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2_wrn40x8_n8_R32_H8": 1.7983e9 * 35_748_708 / 8_388_608}
 
 
+NO_ERROR_ARRAY = False   # --impl2: implementation II of Appendix A.4 (no e array)
+EXACT_COUNT = False      # --exact-count: every mask selects exactly round(B/R) blocks
+
+
 def algorithmic_bytes(w, frac_e_touched):
     """Bytes one step must move: g read; x, (m) read+write; e read+write where touched."""
-    per = 4 + 8 + (8 if w.beta != 0 else 0) + 8 * frac_e_touched
+    per = 4 + 8 + (8 if w.beta != 0 else 0) + (0 if NO_ERROR_ARRAY else 8 * frac_e_touched)
     return w.n_workers * w.d * per
 
 
 def expected_e_fraction(w, is_reset):
-    f = 1.0 - 1.0 / w.R1
+    sel = 1.0 / w.R1 if w.R1 else 0.0
+    f = 1.0 - sel
     if is_reset:
-        f = 1.0 - (1.0 / w.R1) * (1.0 - 1.0 / w.R2)
+        f = 1.0 - sel * (1.0 - 1.0 / w.R2)
     return f
 
 
@@ -189,7 +194,8 @@ def run_workload(w, K, W, dev, rank, world, ring_n=0, with_e2e=True, flush_l2=Fa
 
     # each rank owns one slab of the workload's size, with global block ids
     opt = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
-                 block_begin=rank * w.n_blocks)
+                 block_begin=0 if EXACT_COUNT else rank * w.n_blocks,
+                 flags=(b.FLAG_NO_ERROR_ARRAY if NO_ERROR_ARRAY else 0) | (b.FLAG_EXACT_COUNT if EXACT_COUNT else 0))
     opt.set_x0(synth.x0(w, dev))
     g_bytes = w.n_workers * w.d * 4
     ring_n = ring_n or max(2, min(4, int(6e9 // g_bytes)))
@@ -283,8 +289,13 @@ def main():
     ap.add_argument("--no-others", action="store_true", help="skip the short runs of the other workloads")
     ap.add_argument("--ring", type=int, default=0, help="distinct gradient buffers cycled through")
     ap.add_argument("--d", type=int, default=0, help="override the vector length (small profiling cases)")
+    ap.add_argument("--impl2", action="store_true", help="implementation II (no error array) as the main run")
+    ap.add_argument("--exact-count", action="store_true", help="exact-count GRBS masks as the main run")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    global NO_ERROR_ARRAY, EXACT_COUNT
+    NO_ERROR_ARRAY = bool(args.impl2)
+    EXACT_COUNT = bool(args.exact_count)
 
     from paper_2007_13221_b200 import synth
     w = synth.CONFIGS[args.config]
@@ -318,8 +329,24 @@ def main():
 
     # the other workloads, briefly (single GPU, default invocation only)
     others = None
-    if world == 1 and args.config == 2 and not args.d and not args.no_others:
+    if world == 1 and args.config == 2 and not args.d and not args.no_others and not args.impl2 \
+            and not args.exact_count:
         others = {}
+        EXACT_COUNT = True
+        ro = run_workload(w, 50, 5, dev, rank, world, with_e2e=False)
+        EXACT_COUNT = False
+        others[w.name + " exact-count GRBS (two more small kernels per step)"] = {
+            "steps_per_s": ro["value"], "ms_per_step": ro["ms_per_step"], "steps": 50,
+            "hbm_gbs_step": ro["alg_bytes"] / (ro["ms_per_step"] * 1e-3) / 1e9,
+            "select_kernels_ms_avg": ro["roofline"]["select_kernel_ms_avg"]}
+        NO_ERROR_ARRAY = True
+        ro = run_workload(w, 50, 5, dev, rank, world, with_e2e=False)
+        NO_ERROR_ARRAY = False
+        others[w.name + " implementation II (no error array, 20 B per element-worker)"] = {
+            "steps_per_s": ro["value"], "ms_per_step": ro["ms_per_step"], "steps": 50,
+            "hbm_gbs_step": ro["alg_bytes"] / (ro["ms_per_step"] * 1e-3) / 1e9,
+            "hbm_frac_of_8TBs": ro["alg_bytes"] / (ro["ms_per_step"] * 1e-3) / 1e9 / PEAK_NOMINAL_GBS,
+            "kernel_gbs": ro["roofline"]["achieved"], "kernel_frac_of_measured": ro["roofline"]["frac"]}
         for c in (1, 3, 4, 5):
             wo = synth.CONFIGS[c]
             free, _ = torch.cuda.mem_get_info()
@@ -349,7 +376,9 @@ def main():
             "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "d": w.d, "n_workers": w.n_workers, "block_size": w.block_size,
+            "config": {"workload": w.name + (" implementation II" if args.impl2 else "")
+                       + (" exact-count GRBS" if args.exact_count else ""),
+                       "d": w.d, "n_workers": w.n_workers, "block_size": w.block_size,
                        "R1": w.R1, "R2": w.R2, "H": w.H, "eta": w.eta, "beta": w.beta,
                        "parallelism": f"column slabs x{world}, no collective",
                        "l2": f"inputs larger than L2: {alg_bytes / 1e9:.2f} GB touched per step, "

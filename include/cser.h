@@ -114,6 +114,15 @@ cser_handle cser_create_slab(int64_t d, int32_t n_workers, int32_t block_size,
  *       to rounding.
  */
 #define CSER_FLAG_NO_ERROR_ARRAY 1u
+/*
+ *   CSER_FLAG_EXACT_COUNT  Definition 2 read literally ("picks B/R random blocks"): every
+ *       mask selects exactly k = round(B / R) blocks (halves up; R = 0 gives 0), namely the
+ *       k blocks with the smallest keys (word0, block id), word0 being the same Philox draw
+ *       the default mode thresholds.  Each block is still selected with probability k / B
+ *       and the bytes moved per step no longer fluctuate.  Needs block_begin = 0 and at most
+ *       2^22 blocks.
+ */
+#define CSER_FLAG_EXACT_COUNT 2u
 cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size,
                            uint32_t R1, uint32_t R2, int32_t H,
                            float eta, float beta, uint64_t seed, int64_t block_begin,

@@ -17,5 +17,5 @@ that reduce to textbook SGD, Lemma 1, the mean-model identity, closed forms,
 exact rational brute force, library generators); none is "parity unpinned".
 """
 from .philox import philox4x32_10, philox4_generic          # noqa: F401
-from .grbs import grbs_mask, n_blocks, STREAM_GRAD, STREAM_RESET   # noqa: F401
+from .grbs import grbs_mask, grbs_mask_exact, exact_count, n_blocks, STREAM_GRAD, STREAM_RESET   # noqa: F401
 from .cser import psync, get_p, CSEROracle, CSERImpl2Oracle, CSEAOracle  # noqa: F401

@@ -26,13 +26,15 @@ Readings taken where the paper is silent or inconsistent:
 * On a reset step, line 12 (x <- x - e + e') changes only the reset-selected
   blocks; elsewhere e' = e and the line is the identity, so x is left as is.
 * The two masks of a reset step are drawn independently.
+* ``exact_count=True`` switches the masks to the literal reading of Definition 2
+  (exactly round(B/R) blocks, see ``grbs.grbs_mask_exact``).
 * eta and beta are the float32 values an `float` ABI argument would carry.
 
 The oracle may be evaluated on any subset of columns (``cols``): columns are
 independent given the masks, which always use global block ids.
 """
 import numpy as np
-from .grbs import grbs_mask, n_blocks, STREAM_GRAD, STREAM_RESET
+from .grbs import grbs_mask, grbs_mask_exact, n_blocks, STREAM_GRAD, STREAM_RESET
 
 
 def _mean_over_workers(vc):
@@ -66,7 +68,8 @@ def get_p(m, g, eta, beta):
 
 class _Base:
     def __init__(self, d, n_workers, block_size, R1, R2, H, eta, beta, seed,
-                 dtype=np.float64, cols=None):
+                 dtype=np.float64, cols=None, exact_count=False):
+        self._draw = grbs_mask_exact if exact_count else grbs_mask
         self.d, self.n, self.bs = int(d), int(n_workers), int(block_size)
         self.R1, self.R2, self.H = int(R1), int(R2), int(H)
         self.seed = int(seed)
@@ -105,9 +108,9 @@ class _Base:
             if is_reset:
                 self.mask_r = mr
         else:
-            self.mask_g = grbs_mask(self.seed, t, STREAM_GRAD, self.B, self.R1)
+            self.mask_g = self._draw(self.seed, t, STREAM_GRAD, self.B, self.R1)
             if is_reset:
-                self.mask_r = grbs_mask(self.seed, t, STREAM_RESET, self.B, self.R2)
+                self.mask_r = self._draw(self.seed, t, STREAM_RESET, self.B, self.R2)
         sel_g = self.mask_g[self.block_of_col] != 0
         sel_r = (self.mask_r[self.block_of_col] != 0) if is_reset else None
         return sel_g, sel_r

@@ -36,3 +36,24 @@ def grbs_mask(seed, t, stream, B, R, block_begin=0):
     word0 = philox4x32_10(seed & 0xFFFFFFFF, seed >> 32,
                           b, t & 0xFFFFFFFF, t >> 32, int(stream))[0]
     return (word0.astype(np.uint64) * np.uint64(R) < np.uint64(1 << 32)).astype(np.uint8)
+
+
+def exact_count(B, R):
+    """k of the exact-count reading of Definition 2: round(B / R), halves up; R = 0 gives 0."""
+    if int(R) == 0:
+        return 0
+    return min(int(B), (2 * int(B) + int(R)) // (2 * int(R)))
+
+
+def grbs_mask_exact(seed, t, stream, B, R):
+    """Definition 2 read literally: exactly k = round(B / R) of the B blocks, the k with the
+    smallest keys (word0, block id), word0 being the draw `grbs_mask` thresholds."""
+    k = exact_count(B, R)
+    seed = int(seed) & 0xFFFFFFFFFFFFFFFF
+    t = int(t) & 0xFFFFFFFFFFFFFFFF
+    b = np.arange(B, dtype=np.uint64)
+    word0 = philox4x32_10(seed & 0xFFFFFFFF, seed >> 32, b, t & 0xFFFFFFFF, t >> 32, int(stream))[0]
+    order = np.lexsort((b, word0))                 # by word0, ties by block id
+    mask = np.zeros(B, np.uint8)
+    mask[order[:k]] = 1
+    return mask

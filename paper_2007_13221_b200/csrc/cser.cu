@@ -82,6 +82,113 @@ grbs_mask_kernel(uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r, lon
     (second ? mask_r : mask_g)[b] = sel;
 }
 
+// ------------------------------------------------------------------ exact-count GRBS
+// Definition 2 read literally: exactly k = round(B / R) blocks, those with the k smallest
+// keys (word0, block id).  The k-th smallest key is found in two passes over the B draws
+// with no sorting: a 4096-bin histogram of the top 12 bits of word0 locates the bin that
+// holds it, then the few keys of that bin (about B / 4096) are ranked against each other.
+// Each pass ends in the last CTA to finish (a counter, no waiting), which does the small
+// serial part and re-arms the scratch for the next step.
+constexpr int kExactBins = 4096;
+constexpr int kExactCap = 8192;          // candidate keys kept per mask
+struct ExactScratch {
+    uint32_t hist[2][kExactBins];
+    uint32_t bin[2];                      // bin that holds the k-th smallest key
+    uint32_t k_rem[2];                    // its rank inside that bin (1-based)
+    uint32_t n_cand[2];
+    uint32_t done[2];                     // CTAs finished, one counter per pass
+    unsigned long long thr[2];            // the k-th smallest key
+    unsigned long long cand[2][kExactCap];
+};
+
+__global__ void __launch_bounds__(256)
+grbs_exact_hist_kernel(ExactScratch *__restrict__ X, uint32_t *__restrict__ words, long long B,
+                       uint32_t k0, uint32_t k1, uint32_t t_lo, uint32_t t_hi, uint32_t kg, uint32_t kr,
+                       int n_masks, uint32_t first_which) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx < B * n_masks) {
+        const uint32_t second = idx >= B ? 1u : 0u;
+        const long long b = idx - (second ? B : 0);
+        const uint32_t which = first_which + second;
+        const uint32_t w = philox4x32_10_word0(k0, k1, (uint32_t)b, t_lo, t_hi, which);
+        words[(size_t)which * B + b] = w;
+        atomicAdd(&X->hist[which][w >> 20], 1u);
+    }
+    __shared__ bool last;
+    __shared__ uint32_t part[256];
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = atomicAdd(&X->done[0], 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    for (int q = 0; q < n_masks; ++q) {
+        const uint32_t which = first_which + q;
+        const uint32_t k = which ? kr : kg;
+        volatile uint32_t *h = X->hist[which];
+        constexpr int per = kExactBins / 256;
+        uint32_t loc[per], sum = 0;
+#pragma unroll
+        for (int j = 0; j < per; ++j) { loc[j] = h[threadIdx.x * per + j]; sum += loc[j]; }
+        part[threadIdx.x] = sum;
+        __syncthreads();
+        uint32_t before = 0;                        // draws in bins below this thread's bins
+        for (int j = 0; j < (int)threadIdx.x; ++j) before += part[j];
+        if (k > before && k <= before + sum) {      // the k-th smallest lies in one of my bins
+            uint32_t cum = before;
+#pragma unroll
+            for (int j = 0; j < per; ++j) {
+                if (k > cum && k <= cum + loc[j]) {
+                    X->bin[which] = threadIdx.x * per + j;
+                    X->k_rem[which] = k - cum;
+                }
+                cum += loc[j];
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < per; ++j) h[threadIdx.x * per + j] = 0;   // re-arm for the next step
+        if (threadIdx.x == 0) X->n_cand[which] = 0;
+    }
+    if (threadIdx.x == 0) X->done[0] = 0;
+}
+
+__global__ void __launch_bounds__(256)
+grbs_exact_threshold_kernel(ExactScratch *__restrict__ X, const uint32_t *__restrict__ words, long long B,
+                            int n_masks, uint32_t first_which) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx < B * n_masks) {
+        const uint32_t second = idx >= B ? 1u : 0u;
+        const long long b = idx - (second ? B : 0);
+        const uint32_t which = first_which + second;
+        const uint32_t w = words[(size_t)which * B + b];
+        if ((w >> 20) == X->bin[which]) {
+            const uint32_t at = atomicAdd(&X->n_cand[which], 1u);
+            if (at < (uint32_t)kExactCap) X->cand[which][at] = ((unsigned long long)w << 32) | (uint32_t)b;
+        }
+    }
+    __shared__ bool last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = atomicAdd(&X->done[1], 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    for (int q = 0; q < n_masks; ++q) {
+        const uint32_t which = first_which + q;
+        const uint32_t m = min(*(volatile uint32_t *)&X->n_cand[which], (uint32_t)kExactCap);
+        const uint32_t want = X->k_rem[which] - 1;   // rank (0-based) of the threshold inside the bin
+        const volatile unsigned long long *c = X->cand[which];
+        for (uint32_t i = threadIdx.x; i < m; i += blockDim.x) {
+            const unsigned long long ki = c[i];
+            uint32_t rank = 0;
+            for (uint32_t j = 0; j < m; ++j) rank += c[j] < ki ? 1u : 0u;
+            if (rank == want) X->thr[which] = ki;   // keys are distinct: exactly one writer
+        }
+    }
+    if (threadIdx.x == 0) X->done[1] = 0;
+}
+
 // Per-step block select: one thread per block.  With `draw` it draws the update mask (and,
 // on a reset step, the reset mask) and stores the flags; without it the flags already in
 // mask_g / mask_r are used (injected masks).  Blocks selected by either mask are appended
@@ -92,18 +199,28 @@ __global__ void __launch_bounds__(256)
 grbs_select_kernel(uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r,
                    uint32_t *__restrict__ list, uint32_t *count, uint32_t *count_next, long long B,
                    long long block_begin, uint32_t k0, uint32_t k1, uint32_t t_lo, uint32_t t_hi,
-                   uint32_t R_g, uint32_t R_r, int is_reset, int draw) {
+                   uint32_t R_g, uint32_t R_r, int is_reset, int draw,
+                   const unsigned long long *__restrict__ exact_thr, int exact_g, int exact_r) {
     const long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (b == 0) *count_next = 0;
     bool sg = false, sr = false;
     if (b < B) {
         if (draw) {
             const uint32_t gb = (uint32_t)(block_begin + b);
-            sg = R_g != 0 &&   // R1 = 0: the update compressor keeps nothing (C = 0)
-                 (unsigned long long)philox4x32_10_word0(k0, k1, gb, t_lo, t_hi, 0u) * R_g < (1ull << 32);
+            // R = 0: the compressor keeps nothing (C = 0).  exact_*: keep the blocks whose key
+            // (word0, block id) is not above the k-th smallest key (exact-count GRBS).
+            if (R_g != 0) {
+                const uint32_t w = philox4x32_10_word0(k0, k1, gb, t_lo, t_hi, 0u);
+                sg = exact_g ? ((((unsigned long long)w << 32) | gb) <= exact_thr[0])
+                             : ((unsigned long long)w * R_g < (1ull << 32));
+            }
             mask_g[b] = sg ? 1 : 0;
             if (is_reset) {
-                sr = (unsigned long long)philox4x32_10_word0(k0, k1, gb, t_lo, t_hi, 1u) * R_r < (1ull << 32);
+                if (R_r != 0) {
+                    const uint32_t w = philox4x32_10_word0(k0, k1, gb, t_lo, t_hi, 1u);
+                    sr = exact_r ? ((((unsigned long long)w << 32) | gb) <= exact_thr[1])
+                                 : ((unsigned long long)w * R_r < (1ull << 32));
+                }
                 mask_r[b] = sr ? 1 : 0;
             }
         } else {
@@ -445,6 +562,10 @@ struct cser_ctx {
     uint32_t *sel_count = nullptr;                   // [2] counters, used alternately
     int flip = 0;                                    // which counter the next step uses
     bool walk_all = false;                           // masks were injected: no estimate of the selected count
+    // exact-count GRBS (CSER_FLAG_EXACT_COUNT)
+    bool exact = false;
+    ExactScratch *exact_scratch = nullptr;
+    uint32_t *exact_words = nullptr;                 // [2][B] the step's draws
     // The selected-block kernel and the streaming kernel touch disjoint columns; with an
     // auxiliary stream they run side by side (fork after the select kernel, join after both).
     cudaStream_t aux = nullptr;
@@ -468,13 +589,42 @@ namespace {
 size_t state_elems(const cser_ctx *h) { return (size_t)h->n * (size_t)h->d; }
 
 // GRBS select kernel of iteration h->t.  Leaves the step's counter index in h->flip ^ 1.
+// k of exact-count GRBS: round(B / R), halves up; R = 0 keeps nothing.
+uint32_t exact_k(long long B, uint32_t R) {
+    if (R == 0) return 0;
+    const long long k = (2 * B + R) / (2 * (long long)R);
+    return (uint32_t)(k > B ? B : k);
+}
+
 int launch_select(cser_ctx *h, bool is_reset, bool draw, cudaStream_t s) {
     const unsigned grid = (unsigned)((h->B + 255) / 256);
+    const uint32_t k0 = (uint32_t)(h->seed & 0xffffffffu), k1 = (uint32_t)(h->seed >> 32);
+    const uint32_t t_lo = (uint32_t)(h->t & 0xffffffffu), t_hi = (uint32_t)(h->t >> 32);
+    uint32_t R_g = h->R1, R_r = h->R2;
+    int exact_g = 0, exact_r = 0;
+    if (h->exact && draw) {
+        // k = 0 and k = B need no threshold: they are "nothing" (R = 0) and "everything" (R = 1).
+        const uint32_t kg = exact_k(h->B, h->R1), kr = exact_k(h->B, h->R2);
+        if (kg == 0) R_g = 0; else if (kg >= h->B) R_g = 1; else exact_g = 1;
+        if (is_reset) {
+            if (kr == 0) R_r = 0; else if (kr >= h->B) R_r = 1; else exact_r = 1;
+        }
+        const int n_masks = (exact_g ? 1 : 0) + (exact_r ? 1 : 0);
+        if (n_masks) {
+            const uint32_t first = exact_g ? 0u : 1u;
+            const unsigned g2 = (unsigned)((h->B * n_masks + 255) / 256);
+            grbs_exact_hist_kernel<<<g2, 256, 0, s>>>(h->exact_scratch, h->exact_words, h->B, k0, k1, t_lo,
+                                                      t_hi, kg, kr, n_masks, first);
+            grbs_exact_threshold_kernel<<<g2, 256, 0, s>>>(h->exact_scratch, h->exact_words, h->B, n_masks,
+                                                           first);
+            h->launches += 2;
+            CU_TRY(cudaGetLastError());
+        }
+    }
     grbs_select_kernel<<<grid, 256, 0, s>>>(h->mask_g, h->mask_r, h->sel_list, h->sel_count + h->flip,
-                                            h->sel_count + (h->flip ^ 1), h->B, h->block_begin,
-                                            (uint32_t)(h->seed & 0xffffffffu), (uint32_t)(h->seed >> 32),
-                                            (uint32_t)(h->t & 0xffffffffu), (uint32_t)(h->t >> 32),
-                                            h->R1, h->R2, is_reset ? 1 : 0, draw ? 1 : 0);
+                                            h->sel_count + (h->flip ^ 1), h->B, h->block_begin, k0, k1, t_lo,
+                                            t_hi, R_g, R_r, is_reset ? 1 : 0, draw ? 1 : 0,
+                                            h->exact_scratch ? h->exact_scratch->thr : nullptr, exact_g, exact_r);
     h->launches++;
     CU_TRY(cudaGetLastError());
     h->flip ^= 1;   // the counter just filled is sel_count[h->flip ^ 1] from here on
@@ -605,8 +755,13 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
         fail(CSER_ERR_INVALID, "cser_create: d, n_workers, block_size, R2, H must be positive");
         return nullptr;
     }
-    if (flags & ~(uint32_t)CSER_FLAG_NO_ERROR_ARRAY) {
+    if (flags & ~(uint32_t)(CSER_FLAG_NO_ERROR_ARRAY | CSER_FLAG_EXACT_COUNT)) {
         fail(CSER_ERR_INVALID, "cser_create: unknown flags 0x%x", flags);
+        return nullptr;
+    }
+    if ((flags & CSER_FLAG_EXACT_COUNT) &&
+        (block_begin != 0 || (d + block_size - 1) / block_size > (1ll << 22))) {
+        fail(CSER_ERR_INVALID, "cser_create: exact-count GRBS needs block_begin = 0 and at most 2^22 blocks");
         return nullptr;
     }
     if (!isfinite(eta) || !(beta >= 0.f && beta < 1.f)) {
@@ -637,6 +792,10 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
     if (er == cudaSuccess) er = cudaMemset(h->x, 0, bytes);
     if (er == cudaSuccess && h->e) er = cudaMemset(h->e, 0, bytes);
     if (er == cudaSuccess && h->m) er = cudaMemset(h->m, 0, bytes);
+    h->exact = (flags & CSER_FLAG_EXACT_COUNT) != 0;
+    if (er == cudaSuccess && h->exact) er = cudaMalloc(&h->exact_scratch, sizeof(ExactScratch));
+    if (er == cudaSuccess && h->exact) er = cudaMemset(h->exact_scratch, 0, sizeof(ExactScratch));
+    if (er == cudaSuccess && h->exact) er = cudaMalloc(&h->exact_words, 2 * (size_t)B * sizeof(uint32_t));
     if (er == cudaSuccess) er = cudaMalloc(&h->sel_list, (size_t)B * sizeof(uint32_t));
     if (er == cudaSuccess) er = cudaMalloc(&h->sel_count, 2 * sizeof(uint32_t));
     if (er == cudaSuccess) er = cudaMemset(h->sel_count, 0, 2 * sizeof(uint32_t));
@@ -676,7 +835,7 @@ void cser_destroy(cser_handle h) {
     if (!h) return;
     cudaFree(h->x), cudaFree(h->e), cudaFree(h->m);
     cudaFree(h->mask_g), cudaFree(h->mask_r), cudaFree(h->x0_stage), cudaFree(h->g_stage);
-    cudaFree(h->sel_list), cudaFree(h->sel_count);
+    cudaFree(h->sel_list), cudaFree(h->sel_count), cudaFree(h->exact_scratch), cudaFree(h->exact_words);
     for (auto &ev : h->ev) if (ev) cudaEventDestroy(ev);
     for (auto &ev : h->h_ev) if (ev) cudaEventDestroy(ev);
     for (auto &s : h->hs) if (s) cudaStreamDestroy(s);

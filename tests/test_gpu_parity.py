@@ -14,7 +14,7 @@ import pytest
 import torch
 
 from _golden import read_hand_example
-from oracle import CSEAOracle, CSERImpl2Oracle, CSEROracle, grbs_mask, n_blocks, philox4x32_10, STREAM_GRAD, STREAM_RESET
+from oracle import CSEAOracle, CSERImpl2Oracle, CSEROracle, exact_count, grbs_mask, grbs_mask_exact, n_blocks, philox4x32_10, STREAM_GRAD, STREAM_RESET
 from paper_2007_13221_b200 import binding as b, synth
 
 pytestmark = pytest.mark.gpu
@@ -369,6 +369,44 @@ def test_all_four_mask_combinations_implementation_II():
 
 def test_implementation_II_full_size_headline_workload_on_sampled_blocks():
     _full_size_parity(2, impl2=True)
+
+
+# ------------------------------------------------------------------ exact-count GRBS
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+def test_exact_count_masks_bit_exact_at_every_workload_size(cfg):
+    """d = B (block_size 1... no: one element per block would be slow) - use 4-element blocks, one worker."""
+    w = synth.CONFIGS[cfg]
+    B = w.n_blocks
+    opt = b.CSER(B * 4, 1, 4, w.R1, w.R2, 2, 0.1, 0.0, 77, flags=b.FLAG_EXACT_COUNT)
+    g = torch.zeros((1, B * 4), device=DEV)
+    for t in (1, 2, 3, 4):
+        opt.step(g)
+        mg = opt.state(b.STATE_MASK_G).cpu().numpy()
+        assert int(mg.sum()) == exact_count(B, w.R1)
+        assert np.array_equal(mg, grbs_mask_exact(77, t, STREAM_GRAD, B, w.R1)), (cfg, t)
+        if t % 2 == 0:
+            mr = opt.state(b.STATE_MASK_R).cpu().numpy()
+            assert np.array_equal(mr, grbs_mask_exact(77, t, STREAM_RESET, B, w.R2)), (cfg, t)
+    opt.close()
+
+
+@pytest.mark.parametrize("d,n,bs,R1,R2,H,beta", [(4096 + 40, 8, 256, 4, 4, 4, 0.0), (20_000, 16, 1024, 2, 2, 2, 0.9),
+                                                 (1001, 3, 7, 2, 3, 2, 0.9), (999, 2, 1000, 2, 2, 1, 0.0),
+                                                 (64, 2, 4, 64, 1, 1, 0.9), (262_144 + 4, 8, 512, 32, 32, 8, 0.9)])
+def test_exact_count_mode_equals_its_float32_oracle_exactly(d, n, bs, R1, R2, H, beta):
+    rng = np.random.default_rng(5)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    opt = b.CSER(d, n, bs, R1, R2, H, 0.1, beta, 3, flags=b.FLAG_EXACT_COUNT)
+    ref = CSEROracle(d, n, bs, R1, R2, H, 0.1, beta, 3, dtype=np.float32, exact_count=True)
+    opt.set_x0(torch.from_numpy(x0).to(DEV)), ref.set_x0(x0)
+    for t in range(1, 10):
+        g = rng.standard_normal((n, d)).astype(np.float32)
+        opt.step(torch.from_numpy(g).to(DEV)), ref.step(g)
+        assert np.array_equal(opt.state(b.STATE_MASK_G).cpu().numpy(), ref.mask_g)
+    for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e")) + (((b.STATE_M, "m"),) if beta else ()):
+        assert np.array_equal(opt.state(which).cpu().numpy(), getattr(ref, name)), name
+    opt.close()
+    assert not b.lib().cser_create_ex(100, 2, 4, 2, 2, 2, 0.1, 0.0, 0, 5, b.FLAG_EXACT_COUNT)   # slabs: not supported
 
 
 # ------------------------------------------------------------------ boundary behaviour

@@ -14,7 +14,7 @@ import pytest
 
 from _golden import read_hand_example
 
-from oracle import (CSEAOracle, CSEROracle, CSERImpl2Oracle, grbs_mask, n_blocks, philox4_generic,
+from oracle import (CSEAOracle, CSEROracle, CSERImpl2Oracle, exact_count, grbs_mask, grbs_mask_exact, n_blocks, philox4_generic,
                     philox4x32_10, psync, STREAM_GRAD, STREAM_RESET)
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -425,3 +425,60 @@ def test_cser_pl_with_identity_reset_compressor_is_local_sgd():
             x[:] = x.mean(0)
     assert np.allclose(o.x, x, rtol=1e-12, atol=1e-12)
     assert not o.mask_g.any()
+
+
+# --------------------------------------------------------------------------- exact-count GRBS (Definition 2, literal)
+def test_exact_count_selects_exactly_round_B_over_R_blocks():
+    for B, R in ((4096, 4), (69_822, 32), (24_959, 256), (99_833, 1024), (163_644, 64), (10, 3), (3, 16), (7, 1), (5, 0)):
+        k = exact_count(B, R)
+        assert k == (0 if R == 0 else min(B, int(np.floor(B / R + 0.5))))
+        for t in (1, 2, 9):
+            for stream in (STREAM_GRAD, STREAM_RESET):
+                assert int(grbs_mask_exact(1, t, stream, B, R).sum()) == k
+
+
+def test_exact_count_is_the_k_smallest_draws_by_brute_force():
+    from oracle import philox4x32_10
+    B, R, seed, t = 37, 5, 99, 3
+    words = [int(philox4x32_10(seed, 0, b, t, 0, STREAM_RESET)[0]) for b in range(B)]
+    chosen = sorted(range(B), key=lambda b: (words[b], b))[: exact_count(B, R)]
+    want = np.zeros(B, np.uint8)
+    want[chosen] = 1
+    assert np.array_equal(grbs_mask_exact(seed, t, STREAM_RESET, B, R), want)
+    # whatever is selected has a draw no larger than whatever is not
+    m = grbs_mask_exact(seed, t, STREAM_RESET, B, R).astype(bool)
+    assert max(w for w, s in zip(words, m) if s) <= min(w for w, s in zip(words, m) if not s)
+
+
+def test_exact_count_marginals_are_uniform_and_delta_is_k_over_B():
+    B, R, T = 256, 8, 3000
+    k = exact_count(B, R)
+    freq = np.zeros(B)
+    v = np.random.default_rng(6).standard_normal(B * 4)
+    blk = np.arange(B * 4) // 4
+    ratios = []
+    for t in range(1, T + 1):
+        m = grbs_mask_exact(21, t, STREAM_GRAD, B, R)
+        freq += m
+        if t <= 600:
+            sel = m[blk] != 0
+            ratios.append(((np.where(sel, v, 0) - v) ** 2).sum() / (v**2).sum())
+    z = (freq - T * k / B) / np.sqrt(T * (k / B) * (1 - k / B))
+    assert np.abs(z).max() < 5.0
+    assert abs(np.mean(ratios) - (1 - k / B)) < 0.01
+
+
+def test_exact_count_mode_keeps_the_invariants():
+    n, d, T = 4, 640, 24
+    x0, g = _rand_problem(40, n, d, T)
+    o = CSEROracle(d, n, 8, 4, 2, 3, 0.1, 0.9, 5, exact_count=True)
+    o.set_x0(x0)
+    xbar = x0.astype(np.float64)
+    m = np.zeros((n, d))
+    for gt in g:
+        o.step(gt)
+        m = float(np.float32(0.9)) * m + gt
+        xbar = xbar - (float(np.float32(0.1)) * (float(np.float32(0.9)) * m + gt)).mean(0)
+        assert int(o.mask_g.sum()) == exact_count(o.B, 4)
+        assert np.allclose(o.x.mean(0), xbar, atol=1e-12)
+        assert np.abs((o.x - o.e) - (o.x - o.e)[0]).max() < 1e-12
