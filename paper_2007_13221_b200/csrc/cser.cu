@@ -316,6 +316,10 @@ __device__ __forceinline__ Pack<V> get_p(const Pack<V> &g, Pack<V> &m, float eta
 constexpr int kStepThreads = 256;   // streaming kernel: one CTA = 256 vector columns of one row
 constexpr int kWalkThreads = 128;   // selected-block kernel
 constexpr int kWalkBatch = 4;       // workers whose loads a walking thread keeps in flight
+#ifndef CSER_DENSE_WALK_FRACTION
+#define CSER_DENSE_WALK_FRACTION 0.3
+#endif
+constexpr double kDenseWalkFraction = CSER_DENSE_WALK_FRACTION;   // expected selected share from which the walk is dense
 
 // Selected blocks (1/R of the data): the update needs the mean over workers, so here one
 // thread owns one vector column of a selected block and walks the worker axis.  Threads
@@ -324,22 +328,37 @@ constexpr int kWalkBatch = 4;       // workers whose loads a walking thread keep
 // them (the in-place stores would otherwise keep the compiler from hoisting the next
 // worker's loads), and sums in ascending worker order starting from worker 0's value.
 // This kernel has its own register budget; the streaming kernel stays at 32 registers.
-template <int V, bool MOM, bool RESET, bool ERR>
+// DENSE = false: threads are laid over the listed blocks (few blocks selected).  DENSE =
+// true: one thread per column of the whole range, returning at once if no mask selects its
+// block; used when a large share of the blocks is selected, where walking the columns in
+// their natural order is worth more than the idle threads cost.
+template <int V, bool MOM, bool RESET, bool ERR, bool DENSE>
 __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepParams P) {
     constexpr int U = kWalkBatch;
-    const unsigned long long total = (unsigned long long)(*P.count) * P.bsv;
+    const unsigned long long total =
+        DENSE ? (unsigned long long)(P.c_end - P.c_begin) : (unsigned long long)(*P.count) * P.bsv;
     const long long d = P.d;
     const int n = P.n;
     const float eta = P.eta, beta = P.beta;
     for (unsigned long long f = (unsigned long long)blockIdx.x * kWalkThreads + threadIdx.x; f < total;
          f += (unsigned long long)gridDim.x * kWalkThreads) {
-        const unsigned long long entry = (total <= 0xffffffffull) ? (unsigned long long)((uint32_t)f / P.bsv)
-                                                                  : f / P.bsv;
-        const unsigned blk = P.list[entry];
-        const long long c = (long long)blk * P.bsv + (long long)(f - entry * P.bsv);
-        if (c >= P.cols_total || c < P.c_begin || c >= P.c_end) continue;
+        long long c;
+        unsigned blk;
+        if constexpr (DENSE) {
+            c = P.c_begin + (long long)f;
+            blk = (P.c_end <= 0xffffffffll) ? (uint32_t)c / P.bsv : (unsigned)((unsigned long long)c / P.bsv);
+        } else {
+            const unsigned long long entry =
+                (total <= 0xffffffffull) ? (unsigned long long)((uint32_t)f / P.bsv) : f / P.bsv;
+            blk = P.list[entry];
+            c = (long long)blk * P.bsv + (long long)(f - entry * P.bsv);
+            if (c >= P.cols_total || c < P.c_begin || c >= P.c_end) continue;
+        }
         const bool sg = P.mask_g[blk] != 0;
         const bool sr = RESET ? (P.mask_r[blk] != 0) : false;
+        if constexpr (DENSE) {
+            if (!sg && !sr) continue;
+        }
         const float *__restrict__ g = P.g + c * V;
         float *__restrict__ x = P.x + c * V;
         float *__restrict__ e = ERR ? P.e + c * V : nullptr;
@@ -662,9 +681,14 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
         ws = h->aux;
     }
     const bool err = h->e != nullptr;
+    const bool dense = frac >= kDenseWalkFraction;
+    if (dense) wgrid = wmax;
 #define CSER_LAUNCH_PAIR(MOM_, RESET_, ERR_)                                                            \
     do {                                                                                                \
-        cser_selected_kernel<V, MOM_, RESET_, ERR_><<<(unsigned)wgrid, kWalkThreads, 0, ws>>>(Q);       \
+        if (dense)                                                                                      \
+            cser_selected_kernel<V, MOM_, RESET_, ERR_, true><<<(unsigned)wgrid, kWalkThreads, 0, ws>>>(Q);  \
+        else                                                                                            \
+            cser_selected_kernel<V, MOM_, RESET_, ERR_, false><<<(unsigned)wgrid, kWalkThreads, 0, ws>>>(Q); \
         if (stream_any) cser_stream_kernel<V, MOM_, RESET_, ERR_><<<grid, kStepThreads, 0, s>>>(Q);     \
     } while (0)
 #define CSER_LAUNCH_ERR(MOM_, RESET_)                                                                   \
