@@ -277,6 +277,32 @@ def run_workload(w, K, W, dev, rank, world, ring_n=0, with_e2e=True, flush_l2=Fa
     return out
 
 
+def run_worker_sharded(w, K, W, dev):
+    """The worker-sharded step with this GPU holding all workers (message built, no peer to sum with)."""
+    import torch
+    from paper_2007_13221_b200 import binding as b, synth
+    opt = b.WorkerShardedCSER(w.d, w.n_workers, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed)
+    opt.set_x0(synth.x0(w, dev))
+    ring = [synth.gradients(w, 1 + k, dev) for k in range(3)]
+    for k in range(W):
+        opt.step(ring[k % 3])
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for k in range(K):
+        opt.step(ring[k % 3])
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / K
+    out = {"steps_per_s": 1e3 / ms, "ms_per_step": ms, "steps": K,
+           "message_bytes_plain_step": 4 * b.cser_wshard_message_elems(opt.h, False),
+           "message_bytes_reset_step": 4 * b.cser_wshard_message_elems(opt.h, True)}
+    opt.close()
+    del ring
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -332,6 +358,8 @@ def main():
     if world == 1 and args.config == 2 and not args.d and not args.no_others and not args.impl2 \
             and not args.exact_count:
         others = {}
+        others[w.name + " worker-sharded entry points, one rank holding all workers"] = \
+            run_worker_sharded(w, 50, 5, dev)
         EXACT_COUNT = True
         ro = run_workload(w, 50, 5, dev, rank, world, with_e2e=False)
         EXACT_COUNT = False

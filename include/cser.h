@@ -185,6 +185,32 @@ int cser_grbs_mask(uint64_t seed, uint64_t t, uint32_t which, int64_t block_begi
                    int64_t n_blocks, uint32_t R, uint8_t *mask_out, void *stream);
 
 /*
+ * Worker-sharded deployment (the paper's own setting, Section 3.3: GRBS is compatible with
+ * all-reduce because every worker picks the same blocks).  This GPU holds n_local of the
+ * n_total workers, all d columns.  Masks are exact-count GRBS, so the message length is
+ * known on the host.  One iteration is
+ *     cser_wshard_pack(h, grad, msg, ...)   select, update the unselected blocks, and write
+ *                                           into msg the sum over the LOCAL workers of p on the
+ *                                           update-selected blocks (ascending block order)
+ *                                           followed, on a reset step, by the sum of
+ *                                           e_{t-1/2} on the reset-selected blocks;
+ *     sum msg over all ranks                (the caller's all-reduce, e.g. NCCL);
+ *     cser_wshard_apply(h, msg, ...)        divide by n_total and finish the iteration.
+ * Both PSyncs of a reset step (Algorithm 2 lines 6 and 11) share that one all-reduce.
+ * msg: device, fp32, at least cser_wshard_message_elems(h, reset_step) elements
+ * (reset_step = whether the NEXT iteration t+1 is a multiple of H); a short last block is
+ * padded with zeros.  grad: device fp32 [n_local, d].  With one rank holding all workers the
+ * result equals cser_step's (exact-count masks) bit for bit; across ranks the sum over
+ * workers is associated rank by rank, so results agree to rounding.
+ */
+cser_handle cser_create_wshard(int64_t d, int32_t n_local, int32_t n_total, int32_t block_size,
+                               uint32_t R1, uint32_t R2, int32_t H,
+                               float eta, float beta, uint64_t seed);
+int64_t cser_wshard_message_elems(cser_handle h, int reset_step);   /* -1 if h is not worker-sharded */
+int cser_wshard_pack(cser_handle h, const float *grad, float *msg, size_t msg_elems, void *stream);
+int cser_wshard_apply(cser_handle h, const float *msg, void *stream);
+
+/*
  * Per-kernel timing.  With on != 0, cser_step brackets its mask kernel and its
  * fused step kernel with CUDA events on the launching stream.
  * cser_last_kernel_ms waits for the last step's events and returns both durations

@@ -39,6 +39,15 @@ def lib():
     L.cser_create_slab.argtypes = L.cser_create.argtypes + [c.c_int64]
     L.cser_create_ex.restype = c.c_void_p
     L.cser_create_ex.argtypes = L.cser_create_slab.argtypes + [c.c_uint32]
+    L.cser_create_wshard.restype = c.c_void_p
+    L.cser_create_wshard.argtypes = [c.c_int64, c.c_int32, c.c_int32, c.c_int32, c.c_uint32, c.c_uint32, c.c_int32,
+                                     c.c_float, c.c_float, c.c_uint64]
+    L.cser_wshard_message_elems.restype = c.c_int64
+    L.cser_wshard_message_elems.argtypes = [c.c_void_p, c.c_int]
+    L.cser_wshard_pack.restype = c.c_int
+    L.cser_wshard_pack.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p]
+    L.cser_wshard_apply.restype = c.c_int
+    L.cser_wshard_apply.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p]
     L.cser_destroy.restype = None
     L.cser_destroy.argtypes = [c.c_void_p]
     L.cser_set_x0.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p]
@@ -155,6 +164,26 @@ def cser_launch_count(h):
     return int(lib().cser_launch_count(h))
 
 
+def cser_create_wshard(d, n_local, n_total, block_size, R1, R2, H, eta, beta, seed):
+    h = lib().cser_create_wshard(d, n_local, n_total, block_size, R1, R2, H, eta, beta, seed)
+    if not h:
+        raise CSERError(f"cser_create_wshard failed: {cser_last_error()}")
+    return ctypes.c_void_p(h)
+
+
+def cser_wshard_message_elems(h, reset_step):
+    return int(lib().cser_wshard_message_elems(h, int(bool(reset_step))))
+
+
+def cser_wshard_pack(h, grad, msg, stream=None):
+    assert grad.dtype == torch.float32 and grad.is_contiguous() and grad.is_cuda and msg.dtype == torch.float32
+    _check(lib().cser_wshard_pack(h, _ptr(grad), _ptr(msg), msg.numel(), _stream(stream)), "cser_wshard_pack")
+
+
+def cser_wshard_apply(h, msg, stream=None):
+    _check(lib().cser_wshard_apply(h, _ptr(msg), _stream(stream)), "cser_wshard_apply")
+
+
 class CSER:
     """Convenience owner of one handle (still only marshalling)."""
 
@@ -202,3 +231,40 @@ class CSER:
         out = torch.zeros(1, dtype=torch.int64)
         cser_read_state(self.h, STATE_T, out)
         return int(out.item())
+
+
+class WorkerShardedCSER(CSER):
+    """One rank of the worker-sharded deployment: pack -> all-reduce of the message -> apply.
+
+    torch.distributed is the plumbing for the all-reduce (NCCL between GPUs); with no process
+    group, or a group of one, the message is already the global sum.
+    """
+
+    def __init__(self, d, n_local, n_total, block_size, R1, R2, H, eta, beta, seed=0, group=None):
+        self.d, self.n, self.bs, self.beta = int(d), int(n_local), int(block_size), float(beta)
+        self.H, self.group = int(H), group
+        self.B = (self.d + self.bs - 1) // self.bs
+        self.h = cser_create_wshard(d, n_local, n_total, block_size, R1, R2, H, eta, beta, seed)
+        self.msg = torch.empty(max(1, cser_wshard_message_elems(self.h, True)), dtype=torch.float32,
+                               device="cuda")
+        self._t = 0
+
+    def message_elems(self):
+        """Length of the next step's message."""
+        return cser_wshard_message_elems(self.h, (self._t + 1) % self.H == 0)
+
+    def pack(self, grad):
+        n = self.message_elems()
+        cser_wshard_pack(self.h, grad, self.msg)
+        self._t += 1
+        return self.msg[:n]
+
+    def apply(self):
+        cser_wshard_apply(self.h, self.msg)
+
+    def step(self, grad):
+        import torch.distributed as dist
+        msg = self.pack(grad)
+        if dist.is_available() and dist.is_initialized() and dist.get_world_size(self.group) > 1 and msg.numel():
+            dist.all_reduce(msg, op=dist.ReduceOp.SUM, group=self.group)
+        self.apply()

@@ -551,6 +551,189 @@ __global__ void __launch_bounds__(kStepThreads, 8) cser_stream_kernel(const Step
     if constexpr (ERR) st<V>(P.e + o, ev);
 }
 
+// ------------------------------------------------------------------ worker-sharded step
+// Several GPUs each hold some of the workers (all d columns).  The mean of Algorithm 3 line 7
+// then needs one all-reduce per step.  GRBS makes the compressed vectors directly summable
+// (Section 3.3): every rank selects the same blocks, so each rank packs the sum over its own
+// workers of the selected blocks into a dense message, the messages are summed across ranks,
+// and each rank applies sum / n_total.  The message holds the update-selected blocks in
+// ascending block order and, on a reset step, the reset-selected blocks after them.
+
+// Exclusive scan of the two masks in block order (one CTA): pos_*[b] = selected blocks below b,
+// olist_* = the selected blocks in ascending order.
+__global__ void __launch_bounds__(1024)
+ordered_lists_kernel(const uint8_t *__restrict__ mask_g, const uint8_t *__restrict__ mask_r, long long B,
+                     int is_reset, uint32_t *__restrict__ pos_g, uint32_t *__restrict__ pos_r,
+                     uint32_t *__restrict__ olist_g, uint32_t *__restrict__ olist_r) {
+    __shared__ uint32_t part[2][1024];
+    const long long chunk = (B + blockDim.x - 1) / blockDim.x;
+    const long long b0 = min(B, (long long)threadIdx.x * chunk), b1 = min(B, b0 + chunk);
+    uint32_t cg = 0, cr = 0;
+    for (long long b = b0; b < b1; ++b) {
+        cg += mask_g[b] != 0;
+        if (is_reset) cr += mask_r[b] != 0;
+    }
+    part[0][threadIdx.x] = cg, part[1][threadIdx.x] = cr;
+    __syncthreads();
+    uint32_t og = 0, orr = 0;
+    for (int j = 0; j < (int)threadIdx.x; ++j) og += part[0][j], orr += part[1][j];
+    for (long long b = b0; b < b1; ++b) {
+        pos_g[b] = og;
+        if (mask_g[b]) olist_g[og++] = (uint32_t)b;
+        if (is_reset) {
+            pos_r[b] = orr;
+            if (mask_r[b]) olist_r[orr++] = (uint32_t)b;
+        }
+    }
+}
+
+struct ShardParams {
+    const float *g;
+    float *x, *e, *m;
+    float *msg;                       // [k_g * bs | k_r * bs] floats
+    const uint8_t *mask_g, *mask_r;
+    const uint32_t *pos_g, *olist_g, *olist_r;
+    long long d, cols_total;
+    unsigned bsv, k_g, k_r;
+    int n;                            // local workers
+    float eta, beta, n_total_f;
+};
+
+// Pack: thread f owns vector column (f % bsv) of message block (f / bsv).
+template <int V, bool MOM, bool RESET>
+__global__ void __launch_bounds__(kWalkThreads) wshard_pack_kernel(const ShardParams P) {
+    constexpr int U = kWalkBatch;
+    const unsigned long long total = (unsigned long long)(P.k_g + (RESET ? P.k_r : 0u)) * P.bsv;
+    const long long d = P.d;
+    const int n = P.n;
+    for (unsigned long long f = (unsigned long long)blockIdx.x * kWalkThreads + threadIdx.x; f < total;
+         f += (unsigned long long)gridDim.x * kWalkThreads) {
+        const unsigned entry = (unsigned)(f / P.bsv);
+        const unsigned col = (unsigned)(f - (unsigned long long)entry * P.bsv);
+        const bool r_section = entry >= P.k_g;
+        const unsigned blk = r_section ? P.olist_r[entry - P.k_g] : P.olist_g[entry];
+        const long long c = (long long)blk * P.bsv + col;
+        Pack<V> sum;
+#pragma unroll
+        for (int q = 0; q < V; ++q) sum.v[q] = 0.f;
+        if (c < P.cols_total) {
+            const float *__restrict__ g = P.g + c * V;
+            float *__restrict__ x = P.x + c * V;
+            float *__restrict__ e = P.e + c * V;
+            float *__restrict__ m = MOM ? P.m + c * V : nullptr;
+            if (!r_section) {
+                // update-selected block: sum of the local workers' p, ascending; m updated
+                for (int i0 = 0; i0 < n; i0 += U) {
+                    Pack<V> gv[U], mv[U];
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        if (i0 + u < n) {
+                            const long long o = (long long)(i0 + u) * d;
+                            gv[u] = ld_stream<V>(g + o);
+                            if constexpr (MOM) mv[u] = ld<V>(m + o);
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        if (i0 + u < n) {
+                            const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], P.eta, P.beta);
+                            if constexpr (MOM) st<V>(m + (long long)(i0 + u) * d, mv[u]);
+#pragma unroll
+                            for (int q = 0; q < V; ++q) sum.v[q] = (i0 + u == 0) ? p.v[q] : sum.v[q] + p.v[q];
+                        }
+                    }
+                }
+            } else if (P.mask_g[blk] != 0) {
+                // reset-selected and update-selected: e is unchanged by this step; sum the local e
+                for (int i = 0; i < n; ++i) {
+                    const Pack<V> ev = ld<V>(e + (long long)i * d);
+#pragma unroll
+                    for (int q = 0; q < V; ++q) sum.v[q] = (i == 0) ? ev.v[q] : sum.v[q] + ev.v[q];
+                }
+            } else {
+                // reset-selected only: residual step, store x_{t-1/2} - e_{t-1/2}, zero e, sum e_{t-1/2}
+                for (int i = 0; i < n; ++i) {
+                    const long long o = (long long)i * d;
+                    const Pack<V> gv = ld_stream<V>(g + o);
+                    Pack<V> mv, xv = ld<V>(x + o);
+                    const Pack<V> ev = ld<V>(e + o);
+                    if constexpr (MOM) mv = ld<V>(m + o);
+                    const Pack<V> p = get_p<V, MOM>(gv, mv, P.eta, P.beta);
+                    if constexpr (MOM) st<V>(m + o, mv);
+                    Pack<V> z;
+#pragma unroll
+                    for (int q = 0; q < V; ++q) {
+                        const float xh = xv.v[q] - p.v[q];
+                        const float eh = ev.v[q] - p.v[q];
+                        sum.v[q] = (i == 0) ? eh : sum.v[q] + eh;
+                        xv.v[q] = xh - eh;
+                        z.v[q] = 0.f;
+                    }
+                    st<V>(x + o, xv);
+                    st<V>(e + o, z);
+                }
+            }
+        }
+        st<V>(P.msg + ((size_t)entry * P.bsv + col) * V, sum);   // columns past the end of the vector: zeros
+    }
+}
+
+// Apply the summed message: thread f owns one vector column of one message block.
+template <int V, bool RESET>
+__global__ void __launch_bounds__(kWalkThreads) wshard_apply_kernel(const ShardParams P) {
+    const unsigned long long total = (unsigned long long)(P.k_g + (RESET ? P.k_r : 0u)) * P.bsv;
+    const long long d = P.d;
+    const int n = P.n;
+    for (unsigned long long f = (unsigned long long)blockIdx.x * kWalkThreads + threadIdx.x; f < total;
+         f += (unsigned long long)gridDim.x * kWalkThreads) {
+        const unsigned entry = (unsigned)(f / P.bsv);
+        const unsigned col = (unsigned)(f - (unsigned long long)entry * P.bsv);
+        const bool r_section = entry >= P.k_g;
+        const unsigned blk = r_section ? P.olist_r[entry - P.k_g] : P.olist_g[entry];
+        const long long c = (long long)blk * P.bsv + col;
+        if (c >= P.cols_total) continue;
+        float *__restrict__ x = P.x + c * V;
+        float *__restrict__ e = P.e + c * V;
+        const Pack<V> sv = ld<V>(P.msg + ((size_t)entry * P.bsv + col) * V);
+        Pack<V> mean;
+#pragma unroll
+        for (int q = 0; q < V; ++q) mean.v[q] = sv.v[q] / P.n_total_f;
+        if (!r_section) {
+            if (RESET && P.mask_r[blk] != 0) continue;   // its reset-section thread does both updates
+            for (int i = 0; i < n; ++i) {                // x_i -= mean_k p_k
+                Pack<V> xv = ld<V>(x + (long long)i * d);
+#pragma unroll
+                for (int q = 0; q < V; ++q) xv.v[q] = xv.v[q] - mean.v[q];
+                st<V>(x + (long long)i * d, xv);
+            }
+        } else if (P.mask_g[blk] != 0) {
+            // both masks: x_i = ((x_i - p-bar) - e_i) + e-bar, e_i = 0
+            const Pack<V> sp = ld<V>(P.msg + ((size_t)P.pos_g[blk] * P.bsv + col) * V);
+            for (int i = 0; i < n; ++i) {
+                const long long o = (long long)i * d;
+                Pack<V> xv = ld<V>(x + o);
+                const Pack<V> ev = ld<V>(e + o);
+                Pack<V> z;
+#pragma unroll
+                for (int q = 0; q < V; ++q) {
+                    const float pbar = sp.v[q] / P.n_total_f;
+                    xv.v[q] = ((xv.v[q] - pbar) - ev.v[q]) + mean.v[q];
+                    z.v[q] = 0.f;
+                }
+                st<V>(x + o, xv);
+                st<V>(e + o, z);
+            }
+        } else {
+            for (int i = 0; i < n; ++i) {                // x_i = (x_{t-1/2} - e_{t-1/2}) + e-bar
+                Pack<V> xv = ld<V>(x + (long long)i * d);
+#pragma unroll
+                for (int q = 0; q < V; ++q) xv.v[q] = xv.v[q] + mean.v[q];
+                st<V>(x + (long long)i * d, xv);
+            }
+        }
+    }
+}
+
 // x_i <- x0 for all workers; e, m <- 0
 __global__ void __launch_bounds__(256)
 broadcast_x0_kernel(const float *__restrict__ x0, float *__restrict__ x, float *__restrict__ e,
@@ -581,6 +764,11 @@ struct cser_ctx {
     uint32_t *sel_count = nullptr;                   // [2] counters, used alternately
     int flip = 0;                                    // which counter the next step uses
     bool walk_all = false;                           // masks were injected: no estimate of the selected count
+    // worker-sharded mode (cser_create_wshard): n = local workers, n_total = all ranks' workers
+    int n_total = 0;
+    uint32_t *pos_g = nullptr, *pos_r = nullptr, *olist_g = nullptr, *olist_r = nullptr;
+    bool wshard_open = false;                        // pack done, apply pending
+    bool wshard_reset = false;
     // exact-count GRBS (CSER_FLAG_EXACT_COUNT)
     bool exact = false;
     ExactScratch *exact_scratch = nullptr;
@@ -681,6 +869,20 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
         ws = h->aux;
     }
     const bool err = h->e != nullptr;
+    if (h->n_total > 0) {
+        // worker-sharded: the selected blocks go through pack / all-reduce / apply; only stream here
+        const bool mom_ = h->m != nullptr;
+        if (mom_) {
+            if (is_reset) cser_stream_kernel<V, true, true, true><<<grid, kStepThreads, 0, s>>>(Q);
+            else          cser_stream_kernel<V, true, false, true><<<grid, kStepThreads, 0, s>>>(Q);
+        } else {
+            if (is_reset) cser_stream_kernel<V, false, true, true><<<grid, kStepThreads, 0, s>>>(Q);
+            else          cser_stream_kernel<V, false, false, true><<<grid, kStepThreads, 0, s>>>(Q);
+        }
+        h->launches++;
+        CU_TRY(cudaGetLastError());
+        return CSER_OK;
+    }
     const bool dense = frac >= kDenseWalkFraction;
     if (dense) wgrid = wmax;
 #define CSER_LAUNCH_PAIR(MOM_, RESET_, ERR_)                                                            \
@@ -860,6 +1062,7 @@ void cser_destroy(cser_handle h) {
     cudaFree(h->x), cudaFree(h->e), cudaFree(h->m);
     cudaFree(h->mask_g), cudaFree(h->mask_r), cudaFree(h->x0_stage), cudaFree(h->g_stage);
     cudaFree(h->sel_list), cudaFree(h->sel_count), cudaFree(h->exact_scratch), cudaFree(h->exact_words);
+    cudaFree(h->pos_g), cudaFree(h->pos_r), cudaFree(h->olist_g), cudaFree(h->olist_r);
     for (auto &ev : h->ev) if (ev) cudaEventDestroy(ev);
     for (auto &ev : h->h_ev) if (ev) cudaEventDestroy(ev);
     for (auto &s : h->hs) if (s) cudaStreamDestroy(s);
@@ -895,6 +1098,7 @@ int cser_step(cser_handle h, const float *grad, void *stream) {
     if (int rc = check_handle(h)) return rc;
     if (int rc = check_device_ptr(grad, "cser_step: grad")) return rc;
     if ((uintptr_t)grad % 4 != 0) return fail(CSER_ERR_INVALID, "cser_step: grad is not 4-byte aligned");
+    if (h->n_total > 0) return fail(CSER_ERR_INVALID, "cser_step: worker-sharded handle; use cser_wshard_pack/apply");
     cudaStream_t s = (cudaStream_t)stream;
     const bool is_reset = begin_iteration(h);
     if (h->timing) CU_TRY(cudaEventRecord(h->ev[0], s));
@@ -913,6 +1117,7 @@ int cser_step(cser_handle h, const float *grad, void *stream) {
 int cser_step_host(cser_handle h, const float *grad_host, void *stream) {
     if (int rc = check_handle(h)) return rc;
     if (!grad_host) return fail(CSER_ERR_INVALID, "cser_step_host: grad_host is NULL");
+    if (h->n_total > 0) return fail(CSER_ERR_INVALID, "cser_step_host: worker-sharded handle");
     cudaStream_t s = (cudaStream_t)stream;
     if (!h->g_stage) {
         CU_TRY(cudaMalloc(&h->g_stage, state_elems(h) * sizeof(float)));
@@ -1025,6 +1230,121 @@ int cser_grbs_mask(uint64_t seed, uint64_t t, uint32_t which, int64_t block_begi
         mask_out, mask_out, n_blocks, block_begin, (uint32_t)(seed & 0xffffffffu),
         (uint32_t)(seed >> 32), (uint32_t)(t & 0xffffffffu), (uint32_t)(t >> 32), R, R, 1, which);
     CU_TRY(cudaGetLastError());
+    return CSER_OK;
+}
+
+cser_handle cser_create_wshard(int64_t d, int32_t n_local, int32_t n_total, int32_t block_size, uint32_t R1,
+                               uint32_t R2, int32_t H, float eta, float beta, uint64_t seed) {
+    if (n_local <= 0 || n_total < n_local) {
+        fail(CSER_ERR_INVALID, "cser_create_wshard: need 0 < n_local <= n_total");
+        return nullptr;
+    }
+    cser_ctx *h = cser_create_ex(d, n_local, block_size, R1, R2, H, eta, beta, seed, 0, CSER_FLAG_EXACT_COUNT);
+    if (!h) return nullptr;
+    h->n_total = n_total;
+    cudaError_t er = cudaMalloc(&h->pos_g, (size_t)h->B * sizeof(uint32_t));
+    if (er == cudaSuccess) er = cudaMalloc(&h->pos_r, (size_t)h->B * sizeof(uint32_t));
+    if (er == cudaSuccess) er = cudaMalloc(&h->olist_g, (size_t)h->B * sizeof(uint32_t));
+    if (er == cudaSuccess) er = cudaMalloc(&h->olist_r, (size_t)h->B * sizeof(uint32_t));
+    if (er != cudaSuccess) {
+        fail(er == cudaErrorMemoryAllocation ? CSER_ERR_NOMEM : CSER_ERR_CUDA, "cser_create_wshard: %s",
+             cudaGetErrorString(er));
+        cudaGetLastError();
+        cser_destroy(h);
+        return nullptr;
+    }
+    return h;
+}
+
+int64_t cser_wshard_message_elems(cser_handle h, int reset_step) {
+    if (!h || h->n_total <= 0) return -1;
+    const int64_t kg = exact_k(h->B, h->R1), kr = reset_step ? exact_k(h->B, h->R2) : 0;
+    return (kg + kr) * (int64_t)h->bs;
+}
+
+}  // extern "C"
+
+namespace {
+template <int V>
+int launch_wshard(cser_ctx *h, ShardParams P, bool is_reset, bool pack, cudaStream_t s) {
+    const unsigned long long total = (unsigned long long)(P.k_g + (is_reset ? P.k_r : 0u)) * P.bsv;
+    if (total == 0) return CSER_OK;
+    const unsigned grid = (unsigned)((total + kWalkThreads - 1) / kWalkThreads);
+    const bool mom = h->m != nullptr;
+    if (pack) {
+        if (mom) {
+            if (is_reset) wshard_pack_kernel<V, true, true><<<grid, kWalkThreads, 0, s>>>(P);
+            else          wshard_pack_kernel<V, true, false><<<grid, kWalkThreads, 0, s>>>(P);
+        } else {
+            if (is_reset) wshard_pack_kernel<V, false, true><<<grid, kWalkThreads, 0, s>>>(P);
+            else          wshard_pack_kernel<V, false, false><<<grid, kWalkThreads, 0, s>>>(P);
+        }
+    } else {
+        if (is_reset) wshard_apply_kernel<V, true><<<grid, kWalkThreads, 0, s>>>(P);
+        else          wshard_apply_kernel<V, false><<<grid, kWalkThreads, 0, s>>>(P);
+    }
+    h->launches++;
+    CU_TRY(cudaGetLastError());
+    return CSER_OK;
+}
+
+int wshard_params(cser_ctx *h, const float *grad, float *msg, bool *v4, ShardParams *P) {
+    P->g = grad, P->x = h->x, P->e = h->e, P->m = h->m, P->msg = msg;
+    P->mask_g = h->mask_g, P->mask_r = h->mask_r;
+    P->pos_g = h->pos_g, P->olist_g = h->olist_g, P->olist_r = h->olist_r;
+    P->d = h->d, P->n = h->n;
+    P->k_g = exact_k(h->B, h->R1), P->k_r = exact_k(h->B, h->R2);
+    P->eta = h->eta, P->beta = h->beta, P->n_total_f = (float)h->n_total;
+    *v4 = h->vec4 && ((uintptr_t)msg % 16 == 0) && (!grad || (uintptr_t)grad % 16 == 0);
+    P->bsv = *v4 ? (unsigned)(h->bs / 4) : (unsigned)h->bs;
+    P->cols_total = *v4 ? h->d / 4 : h->d;
+    return CSER_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int cser_wshard_pack(cser_handle h, const float *grad, float *msg, size_t msg_elems, void *stream) {
+    if (int rc = check_handle(h)) return rc;
+    if (h->n_total <= 0) return fail(CSER_ERR_INVALID, "cser_wshard_pack: not a worker-sharded handle");
+    if (h->wshard_open) return fail(CSER_ERR_INVALID, "cser_wshard_pack: previous step was not applied");
+    if (int rc = check_device_ptr(grad, "cser_wshard_pack: grad")) return rc;
+    if (int rc = check_device_ptr(msg, "cser_wshard_pack: msg")) return rc;
+    if (((uintptr_t)grad | (uintptr_t)msg) % 4 != 0)
+        return fail(CSER_ERR_INVALID, "cser_wshard_pack: pointers must be 4-byte aligned");
+    const bool next_reset = ((h->t + 1) % (uint64_t)h->H) == 0;
+    if ((int64_t)msg_elems < cser_wshard_message_elems(h, next_reset))
+        return fail(CSER_ERR_TOO_SMALL, "cser_wshard_pack: message buffer too small");
+    cudaStream_t s = (cudaStream_t)stream;
+    const bool is_reset = begin_iteration(h);
+    if (int rc = launch_select(h, is_reset, true, s)) return rc;
+    ordered_lists_kernel<<<1, 1024, 0, s>>>(h->mask_g, h->mask_r, h->B, is_reset ? 1 : 0, h->pos_g, h->pos_r,
+                                            h->olist_g, h->olist_r);
+    h->launches++;
+    CU_TRY(cudaGetLastError());
+    if (int rc = launch_step(h, grad, 0, h->d, is_reset, s, false)) return rc;   // unselected blocks
+    ShardParams P;
+    bool v4;
+    wshard_params(h, grad, msg, &v4, &P);
+    const int rc = v4 ? launch_wshard<4>(h, P, is_reset, true, s) : launch_wshard<1>(h, P, is_reset, true, s);
+    if (rc) return rc;
+    h->wshard_open = true;
+    h->wshard_reset = is_reset;
+    return CSER_OK;
+}
+
+int cser_wshard_apply(cser_handle h, const float *msg, void *stream) {
+    if (int rc = check_handle(h)) return rc;
+    if (h->n_total <= 0) return fail(CSER_ERR_INVALID, "cser_wshard_apply: not a worker-sharded handle");
+    if (!h->wshard_open) return fail(CSER_ERR_INVALID, "cser_wshard_apply: no packed step pending");
+    if (int rc = check_device_ptr(msg, "cser_wshard_apply: msg")) return rc;
+    ShardParams P;
+    bool v4;
+    wshard_params(h, nullptr, const_cast<float *>(msg), &v4, &P);
+    const int rc = v4 ? launch_wshard<4>(h, P, h->wshard_reset, false, (cudaStream_t)stream)
+                      : launch_wshard<1>(h, P, h->wshard_reset, false, (cudaStream_t)stream);
+    if (rc) return rc;
+    h->wshard_open = false;
     return CSER_OK;
 }
 

@@ -16,3 +16,10 @@ def slab_of_rank(d, block_size, rank, world_size):
     b0 = rank * base + min(rank, extra)
     b1 = b0 + base + (1 if rank < extra else 0)
     return min(b0 * block_size, d), min(b1 * block_size, d), b0
+
+
+def workers_of_rank(n_total, rank, world_size):
+    """(first, count) of the workers `rank` holds in the worker-sharded deployment."""
+    base, extra = divmod(n_total, world_size)
+    first = rank * base + min(rank, extra)
+    return first, base + (1 if rank < extra else 0)

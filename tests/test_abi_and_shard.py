@@ -13,8 +13,8 @@ import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
 
-from oracle import CSEROracle, grbs_mask
-from paper_2007_13221_b200.shard import slab_of_rank
+from oracle import CSEROracle, exact_count, get_p, grbs_mask, grbs_mask_exact
+from paper_2007_13221_b200.shard import slab_of_rank, workers_of_rank
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -127,3 +127,63 @@ def test_two_gloo_ranks_with_column_slabs_equal_the_single_process_result():
     c0, c1, b0 = slab_of_rank(d, 16, 1, 2)
     B = (d + 15) // 16
     assert np.array_equal(grbs_mask(5, 3, 0, B - b0, 4, block_begin=b0), grbs_mask(5, 3, 0, B, 4)[b0:])
+
+
+# ---------------------------------------------------------------- worker-sharded decomposition over gloo
+def _wshard_worker(rank, world, port, q):
+    """Each rank holds some workers, sums its own selected-block values, all-reduces the packed
+    message and applies the mean - the host-side algebra of the worker-sharded step, in NumPy."""
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    n, d, T, x0, g = _problem()
+    bs, R1, R2, H, eta, beta, seed = 16, 4, 2, 3, np.float64(np.float32(0.1)), np.float64(np.float32(0.9)), 5
+    B = (d + bs - 1) // bs
+    first, cnt = workers_of_rank(n, rank, world)
+    x = np.repeat(x0.astype(np.float64)[None, :], cnt, 0)
+    e, m = np.zeros_like(x), np.zeros_like(x)
+    blk = np.arange(d) // bs
+    for t, gt in enumerate(g, 1):
+        is_reset = t % H == 0
+        sg = grbs_mask_exact(seed, t, 0, B, R1)[blk] != 0
+        sr = (grbs_mask_exact(seed, t, 1, B, R2)[blk] != 0) if is_reset else np.zeros(d, bool)
+        p, m = get_p(m, gt[first:first + cnt].astype(np.float64), eta, beta)
+        x_half = np.where(sg[None, :], x, x - p)                    # selected: wait for the mean
+        e_half = np.where(sg[None, :], e, e - p)
+        msg = torch.from_numpy(np.concatenate([p[:, sg].sum(0), e_half[:, sr].sum(0)]))
+        assert msg.numel() == int(sg.sum()) + int(sr.sum())
+        dist.all_reduce(msg)
+        msg = msg.numpy() / n
+        x_half[:, sg] -= msg[: int(sg.sum())][None, :]
+        if is_reset:
+            x_half[:, sr] = (x_half[:, sr] - e_half[:, sr]) + msg[int(sg.sum()):][None, :]
+            e_half[:, sr] = 0
+        x, e = x_half, e_half
+    out = torch.zeros((2, n, d), dtype=torch.float64)
+    out[0, first:first + cnt] = torch.from_numpy(x)
+    out[1, first:first + cnt] = torch.from_numpy(e)
+    dist.all_reduce(out)
+    if rank == 0:
+        q.put(out.numpy())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_worker_sharded_decomposition_over_two_gloo_ranks_matches_the_oracle():
+    n, d, T, x0, g = _problem()
+    ref = CSEROracle(d, n, 16, 4, 2, 3, 0.1, 0.9, 5, dtype=np.float64, exact_count=True)
+    ref.set_x0(x0)
+    for gt in g:
+        ref.step(gt)
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_wshard_worker, args=(r, 2, port, q)) for r in range(2)]
+    [p.start() for p in procs]
+    out = q.get(timeout=120)
+    [p.join(60) for p in procs]
+    assert all(p.exitcode == 0 for p in procs)
+    assert np.allclose(out[0], ref.x, rtol=1e-12, atol=1e-12) and np.allclose(out[1], ref.e, rtol=1e-12, atol=1e-12)
+    assert [workers_of_rank(8, r, 3) for r in range(3)] == [(0, 3), (3, 3), (6, 2)]
