@@ -409,6 +409,67 @@ def test_exact_count_mode_equals_its_float32_oracle_exactly(d, n, bs, R1, R2, H,
     assert not b.lib().cser_create_ex(100, 2, 4, 2, 2, 2, 0.1, 0.0, 0, 5, b.FLAG_EXACT_COUNT)   # slabs: not supported
 
 
+# ------------------------------------------------------------------ more edges
+@pytest.mark.parametrize("d,n,bs,R1,R2,H,beta", [
+    (4, 33, 4, 2, 2, 2, 0.9),          # one vector column, many workers (batches of 4 with a tail of 1)
+    (3, 2, 8, 2, 2, 1, 0.0),           # shorter than one vector column: scalar path, block longer than d
+    (1, 1, 1, 1, 1, 1, 0.9),           # the smallest problem there is
+    (12, 7, 4, 1, 1, 5, 0.0),          # R = 1 without momentum, n not a multiple of the batch
+    (40_000, 64, 128, 16, 8, 2, 0.9),  # many workers
+    (1 << 16, 2, 1 << 16, 2, 2, 2, 0.9),   # a single huge block
+])
+def test_edge_shapes_equal_float32_oracle_exactly(d, n, bs, R1, R2, H, beta):
+    opt, ref = _run_both(d, n, bs, R1, R2, H, 0.1, beta, steps=7)
+    for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e")) + (((b.STATE_M, "m"),) if beta else ()):
+        assert np.array_equal(opt.state(which).cpu().numpy(), getattr(ref, name)), name
+    opt.close()
+
+
+def test_steps_on_a_side_stream_and_kernel_timing_hooks():
+    w = synth.CONFIGS[2].scaled(d=300_000, steps=6)
+    side = torch.cuda.Stream()
+    a = b.CSER(w.d, w.n_workers, w.block_size, 4, 2, 2, w.eta, w.beta, 8)
+    c = b.CSER(w.d, w.n_workers, w.block_size, 4, 2, 2, w.eta, w.beta, 8)
+    x0 = synth.x0(w, DEV)
+    a.set_x0(x0), c.set_x0(x0)
+    grads = [synth.gradients(w, t, DEV) for t in range(1, w.steps + 1)]
+    torch.cuda.synchronize()
+    n0 = b.cser_launch_count(c.h)
+    b.cser_set_timing(c.h, True)
+    for g in grads:
+        a.step(g)
+        with torch.cuda.stream(side):
+            c.step(g)                                   # binding passes torch's current stream
+            sel_ms, step_ms = b.cser_last_kernel_ms(c.h)
+            assert 0.0 < sel_ms < 50.0 and 0.0 < step_ms < 50.0
+    side.synchronize()
+    torch.cuda.synchronize()
+    assert b.cser_launch_count(c.h) - n0 == 3 * len(grads)   # select + selected-block + streaming kernel
+    for which in (b.STATE_X, b.STATE_E, b.STATE_M):
+        assert torch.equal(a.state(which), c.state(which))
+    a.close(), c.close()
+
+
+def test_misaligned_gradient_pointer_takes_the_scalar_path():
+    d, n = 1024, 4
+    rng = np.random.default_rng(3)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    opt = b.CSER(d, n, 64, 2, 2, 2, 0.1, 0.9, 4)
+    ref = CSEROracle(d, n, 64, 2, 2, 2, 0.1, 0.9, 4, dtype=np.float32)
+    opt.set_x0(torch.from_numpy(x0).to(DEV)), ref.set_x0(x0)
+    buf = torch.zeros(n * d + 1, device=DEV)
+    for _ in range(4):
+        g = rng.standard_normal((n, d)).astype(np.float32)
+        view = buf[1:].view(n, d)                      # 4-byte aligned only
+        view.copy_(torch.from_numpy(g))
+        assert view.data_ptr() % 16 == 4
+        b.cser_step(opt.h, view)
+        ref.step(g)
+    assert np.array_equal(opt.state(b.STATE_X).cpu().numpy(), ref.x)
+    assert np.array_equal(opt.state(b.STATE_E).cpu().numpy(), ref.e)
+    opt.close()
+
+
 # ------------------------------------------------------------------ boundary behaviour
 def test_host_gradient_entry_point_equals_device_entry_point():
     w = synth.CONFIGS[2].scaled(d=3_000_000 + 4, steps=10)
