@@ -222,7 +222,7 @@ def run_workload(w, K, W, dev, rank, world, ring_n=0, with_e2e=True, flush_l2=Fa
     # per-kernel durations (CUDA events the library records on the launching stream): the
     # select kernel, then the streaming kernel with the selected-block kernel beside it
     b.cser_set_timing(opt.h, True)
-    k_ms, k_bytes, mask_ms = [], [], []
+    k_ms, k_bytes, mask_ms, k_reset = [], [], [], []
     n_prof = min(K, 4 * w.H if w.H > 1 else 16)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if flush_l2 else None
     for k in range(n_prof):
@@ -232,7 +232,16 @@ def run_workload(w, K, W, dev, rank, world, ring_n=0, with_e2e=True, flush_l2=Fa
         a_ms, s_ms = b.cser_last_kernel_ms(opt.h)
         mask_ms.append(a_ms), k_ms.append(s_ms)
         k_bytes.append(algorithmic_bytes(w, expected_e_fraction(w, opt.t % w.H == 0)))
+        k_reset.append(opt.t % w.H == 0)
     b.cser_set_timing(opt.h, False)
+
+    def stats(sel):
+        v = sorted(ms for ms, r in zip(k_ms, k_reset) if r == sel)
+        by = [bb for bb, r in zip(k_bytes, k_reset) if r == sel]
+        if not v:
+            return None
+        return {"launches": len(v), "ms_mean": sum(v) / len(v), "ms_median": v[len(v) // 2], "ms_min": v[0],
+                "gbs_mean": sum(by) / (sum(v) * 1e-3) / 1e9}
     peak, peak_src = measured_peaks()
     achieved = sum(k_bytes) / (sum(k_ms) * 1e-3) / 1e9
     out["roofline"] = {
@@ -243,6 +252,7 @@ def run_workload(w, K, W, dev, rank, world, ring_n=0, with_e2e=True, flush_l2=Fa
         "algorithmic_bytes_per_launch": sum(k_bytes) / len(k_bytes),
         "kernel_ms_avg": sum(k_ms) / len(k_ms), "select_kernel_ms_avg": sum(mask_ms) / len(mask_ms),
         "launches_timed": len(k_ms), "l2_flushed_between_launches": bool(flush_l2),
+        "plain_steps": stats(False), "reset_steps": stats(True),
     }
     del flush
 
