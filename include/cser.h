@@ -141,7 +141,9 @@ int cser_set_x0(cser_handle h, const float *x0, void *stream);
  * One iteration (Algorithm 2 lines 5-13 / Algorithm 4 lines 5-15) for all workers.
  * grad: device, fp32 [n, d] row-major with leading dimension d; borrowed, read-only,
  * must stay valid and unchanged until the work enqueued on `stream` has finished.
- * Increments t, then enqueues the GRBS mask kernel and the fused step kernel.
+ * Increments t, then enqueues the step kernels (and, beside them, the GRBS select kernel of
+ * the following iteration, whose masks depend only on seed and t; the first step, and a step
+ * after cser_set_x0, cser_write_state(T) or cser_debug_set_masks, runs its own first).
  */
 int cser_step(cser_handle h, const float *grad, void *stream);
 

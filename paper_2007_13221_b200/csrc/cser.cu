@@ -759,10 +759,23 @@ struct cser_ctx {
     float eta = 0.f, beta = 0.f;
     uint64_t seed = 0, t = 0;
     float *x = nullptr, *e = nullptr, *m = nullptr;
+    // Masks and list of the current step (aliases of one of the two buffer sets below).
     uint8_t *mask_g = nullptr, *mask_r = nullptr;
     uint32_t *sel_list = nullptr;                    // [B] blocks selected this step
-    uint32_t *sel_count = nullptr;                   // [2] counters, used alternately
-    int flip = 0;                                    // which counter the next step uses
+    const uint32_t *cur_count = nullptr;             // how many
+    uint8_t *last_mask_r = nullptr;                  // reset mask of the last reset step
+    // The masks of an iteration depend only on (seed, t), so the select kernel of iteration
+    // t + 1 runs during iteration t, beside the step kernels, into the other buffer set.
+    struct SelBuf {
+        uint8_t *mask_g = nullptr, *mask_r = nullptr;
+        uint32_t *list = nullptr;
+    } sb[2];
+    int n_buf = 2, cur = 0;
+    uint32_t *sel_count = nullptr;                   // [3] counters, used in rotation
+    unsigned kseq = 0;                               // select-kernel launches so far
+    bool pre_valid = false;                          // sb[cur ^ 1] holds iteration pre_t
+    uint64_t pre_t = 0;
+    const uint32_t *pre_count = nullptr;
     bool walk_all = false;                           // masks were injected: no estimate of the selected count
     // worker-sharded mode (cser_create_wshard): n = local workers, n_total = all ranks' workers
     int n_total = 0;
@@ -795,7 +808,7 @@ namespace {
 
 size_t state_elems(const cser_ctx *h) { return (size_t)h->n * (size_t)h->d; }
 
-// GRBS select kernel of iteration h->t.  Leaves the step's counter index in h->flip ^ 1.
+// k of exact-count GRBS below; the select launcher follows.
 // k of exact-count GRBS: round(B / R), halves up; R = 0 keeps nothing.
 uint32_t exact_k(long long B, uint32_t R) {
     if (R == 0) return 0;
@@ -803,10 +816,15 @@ uint32_t exact_k(long long B, uint32_t R) {
     return (uint32_t)(k > B ? B : k);
 }
 
-int launch_select(cser_ctx *h, bool is_reset, bool draw, cudaStream_t s) {
+// Select kernel(s) of iteration `t` into buffer set `buf`, on stream s.  Counter k % 3 is
+// used by the k-th launch, which also clears counter (k + 1) % 3; the counter of the launch
+// before (still read by a step kernel that may be running) is left alone.
+int launch_select(cser_ctx *h, int buf, uint64_t t, bool is_reset, bool draw, cudaStream_t s,
+                  const uint32_t **count_out) {
     const unsigned grid = (unsigned)((h->B + 255) / 256);
     const uint32_t k0 = (uint32_t)(h->seed & 0xffffffffu), k1 = (uint32_t)(h->seed >> 32);
-    const uint32_t t_lo = (uint32_t)(h->t & 0xffffffffu), t_hi = (uint32_t)(h->t >> 32);
+    const uint32_t t_lo = (uint32_t)(t & 0xffffffffu), t_hi = (uint32_t)(t >> 32);
+    uint32_t *count = h->sel_count + h->kseq % 3, *count_next = h->sel_count + (h->kseq + 1) % 3;
     uint32_t R_g = h->R1, R_r = h->R2;
     int exact_g = 0, exact_r = 0;
     if (h->exact && draw) {
@@ -828,13 +846,41 @@ int launch_select(cser_ctx *h, bool is_reset, bool draw, cudaStream_t s) {
             CU_TRY(cudaGetLastError());
         }
     }
-    grbs_select_kernel<<<grid, 256, 0, s>>>(h->mask_g, h->mask_r, h->sel_list, h->sel_count + h->flip,
-                                            h->sel_count + (h->flip ^ 1), h->B, h->block_begin, k0, k1, t_lo,
-                                            t_hi, R_g, R_r, is_reset ? 1 : 0, draw ? 1 : 0,
+    grbs_select_kernel<<<grid, 256, 0, s>>>(h->sb[buf].mask_g, h->sb[buf].mask_r, h->sb[buf].list, count,
+                                            count_next, h->B, h->block_begin, k0, k1, t_lo, t_hi, R_g, R_r,
+                                            is_reset ? 1 : 0, draw ? 1 : 0,
                                             h->exact_scratch ? h->exact_scratch->thr : nullptr, exact_g, exact_r);
     h->launches++;
     CU_TRY(cudaGetLastError());
-    h->flip ^= 1;   // the counter just filled is sel_count[h->flip ^ 1] from here on
+    h->kseq++;
+    *count_out = count;
+    return CSER_OK;
+}
+
+// Make buffer set `buf` (with its list counter) the current step's.
+void activate_selection(cser_ctx *h, int buf, const uint32_t *count, bool is_reset) {
+    h->cur = buf;
+    h->mask_g = h->sb[buf].mask_g, h->mask_r = h->sb[buf].mask_r, h->sel_list = h->sb[buf].list;
+    h->cur_count = count;
+    if (is_reset) h->last_mask_r = h->sb[buf].mask_r;
+}
+
+// Masks and list for iteration h->t: take the prefetched ones if they are for this iteration,
+// else run the select kernel now on stream s.
+int select_for_iteration(cser_ctx *h, bool is_reset, cudaStream_t s) {
+    if (h->pre_valid && h->pre_t == h->t && !h->masks_injected) {
+        activate_selection(h, h->cur ^ 1, h->pre_count, is_reset);
+        h->pre_valid = false;
+        h->walk_all = false;
+        return CSER_OK;
+    }
+    const int nb = h->n_buf == 2 ? (h->cur ^ 1) : 0;
+    const uint32_t *count = nullptr;
+    if (int rc = launch_select(h, nb, h->t, is_reset, !h->masks_injected, s, &count)) return rc;
+    activate_selection(h, nb, count, is_reset);
+    h->pre_valid = false;
+    h->walk_all = h->masks_injected;
+    h->masks_injected = false;
     return CSER_OK;
 }
 
@@ -910,6 +956,15 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     h->launches += stream_any ? 2 : 1;
     CU_TRY(cudaGetLastError());
     if (fork) {
+        if (h->n_buf == 2) {
+            // next iteration's select kernel, off the critical path
+            const uint64_t t_next = h->t + 1;
+            if (int rc = launch_select(h, h->cur ^ 1, t_next, (t_next % (uint64_t)h->H) == 0, true, h->aux,
+                                       &h->pre_count))
+                return rc;
+            h->pre_valid = true;
+            h->pre_t = t_next;
+        }
         CU_TRY(cudaEventRecord(h->ev_join, h->aux));
         CU_TRY(cudaStreamWaitEvent(s, h->ev_join, 0));
     }
@@ -922,7 +977,7 @@ int launch_step(cser_ctx *h, const float *grad, long long col0, long long col1, 
     StepParams P;
     P.g = grad, P.x = h->x, P.e = h->e, P.m = h->m;
     P.mask_g = h->mask_g, P.mask_r = h->mask_r;
-    P.list = h->sel_list, P.count = h->sel_count + (h->flip ^ 1);
+    P.list = h->sel_list, P.count = h->cur_count;
     P.tiles = 0;
     P.d = h->d, P.n = h->n;
     P.eta = h->eta, P.beta = h->beta, P.n_f = (float)h->n;
@@ -1013,8 +1068,13 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
     const bool with_e = !(flags & CSER_FLAG_NO_ERROR_ARRAY);
     if (er == cudaSuccess && with_e) er = cudaMalloc(&h->e, bytes);
     if (er == cudaSuccess && beta != 0.f) er = cudaMalloc(&h->m, bytes);
-    if (er == cudaSuccess) er = cudaMalloc(&h->mask_g, (size_t)B);
-    if (er == cudaSuccess) er = cudaMalloc(&h->mask_r, (size_t)B);
+    for (auto &sb : h->sb) {
+        if (er == cudaSuccess) er = cudaMalloc(&sb.mask_g, (size_t)B);
+        if (er == cudaSuccess) er = cudaMalloc(&sb.mask_r, (size_t)B);
+        if (er == cudaSuccess) er = cudaMalloc(&sb.list, (size_t)B * sizeof(uint32_t));
+        if (er == cudaSuccess) er = cudaMemset(sb.mask_g, 0, (size_t)B);
+        if (er == cudaSuccess) er = cudaMemset(sb.mask_r, 0, (size_t)B);
+    }
     if (er == cudaSuccess) er = cudaMemset(h->x, 0, bytes);
     if (er == cudaSuccess && h->e) er = cudaMemset(h->e, 0, bytes);
     if (er == cudaSuccess && h->m) er = cudaMemset(h->m, 0, bytes);
@@ -1022,11 +1082,9 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
     if (er == cudaSuccess && h->exact) er = cudaMalloc(&h->exact_scratch, sizeof(ExactScratch));
     if (er == cudaSuccess && h->exact) er = cudaMemset(h->exact_scratch, 0, sizeof(ExactScratch));
     if (er == cudaSuccess && h->exact) er = cudaMalloc(&h->exact_words, 2 * (size_t)B * sizeof(uint32_t));
-    if (er == cudaSuccess) er = cudaMalloc(&h->sel_list, (size_t)B * sizeof(uint32_t));
-    if (er == cudaSuccess) er = cudaMalloc(&h->sel_count, 2 * sizeof(uint32_t));
-    if (er == cudaSuccess) er = cudaMemset(h->sel_count, 0, 2 * sizeof(uint32_t));
-    if (er == cudaSuccess) er = cudaMemset(h->mask_g, 0, (size_t)B);
-    if (er == cudaSuccess) er = cudaMemset(h->mask_r, 0, (size_t)B);
+    if (er == cudaSuccess) er = cudaMalloc(&h->sel_count, 3 * sizeof(uint32_t));
+    if (er == cudaSuccess) er = cudaMemset(h->sel_count, 0, 3 * sizeof(uint32_t));
+    if (er == cudaSuccess) activate_selection(h, 0, h->sel_count, true);
     for (int k = 0; k < 3 && er == cudaSuccess; ++k) er = cudaEventCreate(&h->ev[k]);
     if (er == cudaSuccess) {
         int lo = 0, hi = 0;   // hi = numerically lowest = highest priority
@@ -1060,8 +1118,9 @@ cser_handle cser_create(int64_t d, int32_t n_workers, int32_t block_size, uint32
 void cser_destroy(cser_handle h) {
     if (!h) return;
     cudaFree(h->x), cudaFree(h->e), cudaFree(h->m);
-    cudaFree(h->mask_g), cudaFree(h->mask_r), cudaFree(h->x0_stage), cudaFree(h->g_stage);
-    cudaFree(h->sel_list), cudaFree(h->sel_count), cudaFree(h->exact_scratch), cudaFree(h->exact_words);
+    for (auto &sb : h->sb) cudaFree(sb.mask_g), cudaFree(sb.mask_r), cudaFree(sb.list);
+    cudaFree(h->x0_stage), cudaFree(h->g_stage);
+    cudaFree(h->sel_count), cudaFree(h->exact_scratch), cudaFree(h->exact_words);
     cudaFree(h->pos_g), cudaFree(h->pos_r), cudaFree(h->olist_g), cudaFree(h->olist_r);
     for (auto &ev : h->ev) if (ev) cudaEventDestroy(ev);
     for (auto &ev : h->h_ev) if (ev) cudaEventDestroy(ev);
@@ -1091,6 +1150,7 @@ int cser_set_x0(cser_handle h, const float *x0, void *stream) {
     CU_TRY(cudaGetLastError());
     h->t = 0;
     h->masks_injected = false;
+    h->pre_valid = false;
     return CSER_OK;
 }
 
@@ -1102,9 +1162,7 @@ int cser_step(cser_handle h, const float *grad, void *stream) {
     cudaStream_t s = (cudaStream_t)stream;
     const bool is_reset = begin_iteration(h);
     if (h->timing) CU_TRY(cudaEventRecord(h->ev[0], s));
-    if (int rc = launch_select(h, is_reset, !h->masks_injected, s)) return rc;
-    h->walk_all = h->masks_injected;
-    h->masks_injected = false;
+    if (int rc = select_for_iteration(h, is_reset, s)) return rc;
     if (h->timing) CU_TRY(cudaEventRecord(h->ev[1], s));
     if (int rc = launch_step(h, grad, 0, h->d, is_reset, s, true)) return rc;
     if (h->timing) {
@@ -1126,9 +1184,7 @@ int cser_step_host(cser_handle h, const float *grad_host, void *stream) {
     }
     const bool is_reset = begin_iteration(h);
     // masks first, on the caller's stream; both internal streams start after them
-    if (int rc = launch_select(h, is_reset, !h->masks_injected, s)) return rc;
-    h->walk_all = h->masks_injected;
-    h->masks_injected = false;
+    if (int rc = select_for_iteration(h, is_reset, s)) return rc;
     CU_TRY(cudaEventRecord(h->h_ev[0], s));
     CU_TRY(cudaStreamWaitEvent(h->hs[0], h->h_ev[0], 0));
     CU_TRY(cudaStreamWaitEvent(h->hs[1], h->h_ev[0], 0));
@@ -1166,7 +1222,7 @@ static int state_piece(cser_ctx *h, int which, void **ptr, size_t *bytes) {
             *ptr = h->m, *bytes = state_elems(h) * sizeof(float);
             return CSER_OK;
         case CSER_STATE_MASK_G: *ptr = h->mask_g, *bytes = (size_t)h->B; return CSER_OK;
-        case CSER_STATE_MASK_R: *ptr = h->mask_r, *bytes = (size_t)h->B; return CSER_OK;
+        case CSER_STATE_MASK_R: *ptr = h->last_mask_r, *bytes = (size_t)h->B; return CSER_OK;
         case CSER_STATE_T: *ptr = nullptr, *bytes = sizeof(uint64_t); return CSER_OK;
         default: return fail(CSER_ERR_INVALID, "unknown state id %d", which);
     }
@@ -1200,6 +1256,7 @@ int cser_write_state(cser_handle h, int which, const void *src, size_t bytes, vo
         return fail(CSER_ERR_TOO_SMALL, "cser_write_state: need exactly %zu bytes, got %zu", want, bytes);
     if (which == CSER_STATE_T) {
         CU_TRY(cudaMemcpy(&h->t, src, sizeof(uint64_t), cudaMemcpyDefault));
+        h->pre_valid = false;
         return CSER_OK;
     }
     CU_TRY(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, (cudaStream_t)stream));
@@ -1213,8 +1270,9 @@ int cser_debug_set_masks(cser_handle h, const uint8_t *g_mask, const uint8_t *r_
     if (next_is_reset && !r_mask)
         return fail(CSER_ERR_INVALID, "cser_debug_set_masks: next step resets, r_mask is NULL");
     cudaStream_t s = (cudaStream_t)stream;
-    CU_TRY(cudaMemcpyAsync(h->mask_g, g_mask, (size_t)h->B, cudaMemcpyDefault, s));
-    if (r_mask) CU_TRY(cudaMemcpyAsync(h->mask_r, r_mask, (size_t)h->B, cudaMemcpyDefault, s));
+    const int nb = h->n_buf == 2 ? (h->cur ^ 1) : 0;   // the set the next step's select kernel reads
+    CU_TRY(cudaMemcpyAsync(h->sb[nb].mask_g, g_mask, (size_t)h->B, cudaMemcpyDefault, s));
+    if (r_mask) CU_TRY(cudaMemcpyAsync(h->sb[nb].mask_r, r_mask, (size_t)h->B, cudaMemcpyDefault, s));
     h->masks_injected = true;
     return CSER_OK;
 }
@@ -1317,7 +1375,7 @@ int cser_wshard_pack(cser_handle h, const float *grad, float *msg, size_t msg_el
         return fail(CSER_ERR_TOO_SMALL, "cser_wshard_pack: message buffer too small");
     cudaStream_t s = (cudaStream_t)stream;
     const bool is_reset = begin_iteration(h);
-    if (int rc = launch_select(h, is_reset, true, s)) return rc;
+    if (int rc = select_for_iteration(h, is_reset, s)) return rc;
     ordered_lists_kernel<<<1, 1024, 0, s>>>(h->mask_g, h->mask_r, h->B, is_reset ? 1 : 0, h->pos_g, h->pos_r,
                                             h->olist_g, h->olist_r);
     h->launches++;
@@ -1376,7 +1434,7 @@ int64_t cser_launch_count(cser_handle h) { return h ? h->launches : 0; }
 // masks, the list of selected blocks and two list counters.  For callers that must not
 // allocate, that scratch lives here: a fixed array that every GPU which loads this
 // library keeps until the process exits.  Layout (bytes): update mask [0, MAXB), reset
-// mask [MAXB, 2 MAXB), list of uint32 [2 MAXB, 6 MAXB), two uint32 counters after it.
+// mask [MAXB, 2 MAXB), list of uint32 [2 MAXB, 6 MAXB), three uint32 counters after it.
 // Static device memory starts zeroed, which is the state the counters need.
 constexpr size_t kNoallocMaxB = CSER_NOALLOC_MAX_BLOCKS;
 constexpr size_t kNoallocBytes = 6 * kNoallocMaxB + 256;
@@ -1389,7 +1447,7 @@ constexpr int kNoallocMaxDevices = 64;
 // code the array's name is only a handle for the runtime, never an address a kernel may
 // be given; cudaGetSymbolAddress translates it for the device that is current.
 uint8_t *g_noalloc_addr[kNoallocMaxDevices] = {};
-int g_noalloc_flip[kNoallocMaxDevices] = {};      // which counter the next call uses
+unsigned g_noalloc_kseq[kNoallocMaxDevices] = {};  // select launches so far: picks the list counter
 
 int noalloc_scratch(int device, uint8_t **out) {
     if (device < 0 || device >= kNoallocMaxDevices)
@@ -1443,10 +1501,11 @@ extern "C" int cser_step_noalloc(int64_t d, int32_t n_workers, int32_t block_siz
     c.eta = eta, c.beta = beta, c.seed = seed, c.B = B, c.block_begin = 0;
     c.t = t;
     c.x = x, c.e = e, c.m = (beta != 0.f) ? m : nullptr;
-    c.mask_g = scratch, c.mask_r = scratch + kNoallocMaxB;
-    c.sel_list = reinterpret_cast<uint32_t *>(scratch + 2 * kNoallocMaxB);
+    c.n_buf = 1;
+    c.sb[0].mask_g = scratch, c.sb[0].mask_r = scratch + kNoallocMaxB;
+    c.sb[0].list = reinterpret_cast<uint32_t *>(scratch + 2 * kNoallocMaxB);
     c.sel_count = reinterpret_cast<uint32_t *>(scratch + 6 * kNoallocMaxB);
-    c.flip = g_noalloc_flip[c.device];
+    c.kseq = g_noalloc_kseq[c.device];
     c.vec4 = (d % 4 == 0) && (block_size % 4 == 0) &&
              (((uintptr_t)x | (uintptr_t)e | (uintptr_t)c.m) % 16 == 0);
     const bool is_reset = (t % (uint64_t)H) == 0;
@@ -1454,8 +1513,8 @@ extern "C" int cser_step_noalloc(int64_t d, int32_t n_workers, int32_t block_siz
     // The select kernel rewrites every mask entry and list entry the step kernel reads and
     // clears the counter the next call will use, so nothing an earlier call left in the
     // array is ever used and nothing has to be cleared between calls.
-    const int rc = launch_select(&c, is_reset, true, s);
-    g_noalloc_flip[c.device] = c.flip;
+    const int rc = select_for_iteration(&c, is_reset, s);
+    g_noalloc_kseq[c.device] = c.kseq;
     if (rc) return rc;
     return launch_step(&c, grad, 0, d, is_reset, s);
 }
