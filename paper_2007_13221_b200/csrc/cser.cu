@@ -808,7 +808,6 @@ namespace {
 
 size_t state_elems(const cser_ctx *h) { return (size_t)h->n * (size_t)h->d; }
 
-// k of exact-count GRBS below; the select launcher follows.
 // k of exact-count GRBS: round(B / R), halves up; R = 0 keeps nothing.
 uint32_t exact_k(long long B, uint32_t R) {
     if (R == 0) return 0;
@@ -956,17 +955,18 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     h->launches += stream_any ? 2 : 1;
     CU_TRY(cudaGetLastError());
     if (fork) {
+        int rc = CSER_OK;
         if (h->n_buf == 2) {
             // next iteration's select kernel, off the critical path
             const uint64_t t_next = h->t + 1;
-            if (int rc = launch_select(h, h->cur ^ 1, t_next, (t_next % (uint64_t)h->H) == 0, true, h->aux,
-                                       &h->pre_count))
-                return rc;
-            h->pre_valid = true;
+            rc = launch_select(h, h->cur ^ 1, t_next, (t_next % (uint64_t)h->H) == 0, true, h->aux,
+                               &h->pre_count);
+            h->pre_valid = rc == CSER_OK;
             h->pre_t = t_next;
         }
-        CU_TRY(cudaEventRecord(h->ev_join, h->aux));
+        CU_TRY(cudaEventRecord(h->ev_join, h->aux));      // join even if the prefetch could not be launched
         CU_TRY(cudaStreamWaitEvent(s, h->ev_join, 0));
+        return rc;
     }
     return CSER_OK;
 }
