@@ -145,6 +145,66 @@ def oracle_sample_rate(w, target_seconds=15.0, sample_cols=1 << 18):
     return rate, desc, 1, el
 
 
+def oracle_all_cores(w, seconds=10.0):
+    """The same oracle with the columns split over all host cores: one process per core, each
+    timing its own slab of whole blocks at the same moment.  Returns (steps/s, description, cores)."""
+    import subprocess
+    cores = os.cpu_count() or 1
+    procs = [subprocess.Popen([sys.executable, os.path.abspath(__file__), "--config", str(w_index(w)),
+                               "--oracle-slab", str(k), "--oracle-seconds", str(seconds)] +
+                              (["--d", str(w.d)] if w.d != base_config(w).d else []),
+                              stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True,
+                              env={**os.environ, "OMP_NUM_THREADS": "1", "MKL_NUM_THREADS": "1",
+                                   "CUDA_VISIBLE_DEVICES": ""})
+             for k in range(cores)]
+    total, ok = 0.0, 0
+    for p in procs:
+        out, _ = p.communicate(timeout=600)
+        try:
+            total += float(json.loads(out.strip().splitlines()[-1])["rate"])
+            ok += 1
+        except Exception:
+            pass
+    desc = (f"{ok} processes, one per core, each stepping the float64 NumPy oracle on its own 65,536-column slab "
+            f"of {w.name} for {seconds:.0f} s at the same time; rates (scaled to the full vector) added")
+    return total, desc, ok
+
+
+def base_config(w):
+    from paper_2007_13221_b200 import synth
+    return synth.CONFIGS[w_index(w)]
+
+
+def w_index(w):
+    from paper_2007_13221_b200 import synth
+    for k, c in synth.CONFIGS.items():
+        if w.name.startswith(c.name):
+            return k
+    raise ValueError(w.name)
+
+
+def oracle_slab_worker(w, slab, seconds):
+    """Child of oracle_all_cores: times the oracle on columns [slab * 65536, (slab + 1) * 65536)."""
+    import numpy as np
+    from oracle import CSEROracle
+    from paper_2007_13221_b200 import synth
+    width = 65536 // w.block_size * w.block_size
+    c0 = (slab * width) % max(width, (w.d - width) // w.block_size * w.block_size)
+    cols = np.arange(c0, min(c0 + width, w.d))
+    ws = w.scaled(cols.size)
+    ref = CSEROracle(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
+                     dtype=np.float64, cols=cols)
+    ref.set_x0(synth.x0(ws, "cpu").numpy())
+    grads = [synth.gradients(ws, t, "cpu").numpy() for t in range(1, 4)]
+    ref.step(grads[0])
+    n_steps, t0 = 0, time.perf_counter()
+    while time.perf_counter() - t0 < seconds:
+        ref.step(grads[n_steps % 3])
+        n_steps += 1
+    el = time.perf_counter() - t0
+    print(json.dumps({"rate": n_steps / el * (cols.size / w.d)}))
+
+
 def run_reference(args, w):
     """--impl reference: the oracle, timed on the host cores, same metric and workload."""
     rank = int(os.environ.get("RANK", "0"))
@@ -327,6 +387,8 @@ def main():
     ap.add_argument("--d", type=int, default=0, help="override the vector length (small profiling cases)")
     ap.add_argument("--impl2", action="store_true", help="implementation II (no error array) as the main run")
     ap.add_argument("--exact-count", action="store_true", help="exact-count GRBS masks as the main run")
+    ap.add_argument("--oracle-slab", type=int, default=-1, help=argparse.SUPPRESS)
+    ap.add_argument("--oracle-seconds", type=float, default=10.0, help=argparse.SUPPRESS)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     global NO_ERROR_ARRAY, EXACT_COUNT
@@ -337,6 +399,9 @@ def main():
     w = synth.CONFIGS[args.config]
     if args.d:
         w = w.scaled(args.d)
+    if args.oracle_slab >= 0:
+        oracle_slab_worker(w, args.oracle_slab, args.oracle_seconds)
+        return
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -408,6 +473,8 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         rate, desc, cores, _ = oracle_sample_rate(w)
         cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+        rate_all, desc_all, cores_all = oracle_all_cores(w)
+        cpu["all_cores"] = {"value": rate_all, "unit": UNIT, "cores": cores_all, "sample": desc_all}
 
     if rank == 0:
         line = {
