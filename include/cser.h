@@ -165,6 +165,20 @@ int cser_step_host(cser_handle h, const float *grad_host, void *stream);
 int cser_read_state(cser_handle h, int which, void *dst, size_t dst_bytes, void *stream);
 
 /*
+ * Copy columns [col_begin, col_begin + col_count) of x, e or m, for all workers, into dst
+ * (host or device) as a dense fp32 [n, col_count] array; enqueued on `stream`.  For looking
+ * at part of a state that is too large to copy whole.
+ */
+int cser_read_columns(cser_handle h, int which, int64_t col_begin, int64_t col_count,
+                      float *dst, size_t dst_elems, void *stream);
+
+/*
+ * Learning rate eta for the following steps (the schedules of Section 5.1 change it between
+ * steps; Algorithms 2 and 4 take it as given).  Takes effect with the next cser_step.
+ */
+int cser_set_lr(cser_handle h, float eta);
+
+/*
  * Restore one piece of state from src (host or device) - the inverse of
  * cser_read_state, for checkpoint/resume.  `bytes` must be exactly the piece's size.
  * Masks cannot be written (use cser_debug_set_masks).

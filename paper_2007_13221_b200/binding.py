@@ -55,6 +55,10 @@ def lib():
     L.cser_step_host.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p]
     L.cser_read_state.argtypes = [c.c_void_p, c.c_int, c.c_void_p, c.c_size_t, c.c_void_p]
     L.cser_write_state.argtypes = [c.c_void_p, c.c_int, c.c_void_p, c.c_size_t, c.c_void_p]
+    L.cser_read_columns.restype = c.c_int
+    L.cser_read_columns.argtypes = [c.c_void_p, c.c_int, c.c_int64, c.c_int64, c.c_void_p, c.c_size_t, c.c_void_p]
+    L.cser_set_lr.restype = c.c_int
+    L.cser_set_lr.argtypes = [c.c_void_p, c.c_float]
     L.cser_debug_set_masks.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
     L.cser_grbs_mask.argtypes = [c.c_uint64, c.c_uint64, c.c_uint32, c.c_int64, c.c_int64, c.c_uint32,
                                  c.c_void_p, c.c_void_p]
@@ -125,6 +129,16 @@ def cser_step_host(h, grad_host, stream=None):
 def cser_read_state(h, which, dst, stream=None):
     _check(lib().cser_read_state(h, which, _ptr(dst), dst.numel() * dst.element_size(), _stream(stream)),
            "cser_read_state")
+
+
+def cser_read_columns(h, which, col_begin, col_count, dst, stream=None):
+    assert dst.dtype == torch.float32 and dst.is_contiguous()
+    _check(lib().cser_read_columns(h, which, col_begin, col_count, _ptr(dst), dst.numel(), _stream(stream)),
+           "cser_read_columns")
+
+
+def cser_set_lr(h, eta):
+    _check(lib().cser_set_lr(h, eta), "cser_set_lr")
 
 
 def cser_write_state(h, which, src, stream=None):

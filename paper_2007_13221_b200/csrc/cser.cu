@@ -1244,6 +1244,33 @@ int cser_read_state(cser_handle h, int which, void *dst, size_t dst_bytes, void 
     return CSER_OK;
 }
 
+int cser_read_columns(cser_handle h, int which, int64_t col_begin, int64_t col_count, float *dst,
+                      size_t dst_elems, void *stream) {
+    if (int rc = check_handle(h)) return rc;
+    if (!dst) return fail(CSER_ERR_INVALID, "cser_read_columns: dst is NULL");
+    if (which != CSER_STATE_X && which != CSER_STATE_E && which != CSER_STATE_M)
+        return fail(CSER_ERR_INVALID, "cser_read_columns: which must be x, e or m");
+    if (col_begin < 0 || col_count < 0 || col_begin + col_count > h->d)
+        return fail(CSER_ERR_INVALID, "cser_read_columns: column range outside [0, d)");
+    void *src;
+    size_t bytes;
+    if (int rc = state_piece(h, which, &src, &bytes)) return rc;
+    if (dst_elems < (size_t)h->n * (size_t)col_count)
+        return fail(CSER_ERR_TOO_SMALL, "cser_read_columns: need %zu elements", (size_t)h->n * (size_t)col_count);
+    if (col_count == 0) return CSER_OK;
+    CU_TRY(cudaMemcpy2DAsync(dst, (size_t)col_count * sizeof(float), static_cast<float *>(src) + col_begin,
+                             (size_t)h->d * sizeof(float), (size_t)col_count * sizeof(float), (size_t)h->n,
+                             cudaMemcpyDefault, (cudaStream_t)stream));
+    return CSER_OK;
+}
+
+int cser_set_lr(cser_handle h, float eta) {
+    if (int rc = check_handle(h)) return rc;
+    if (!isfinite(eta)) return fail(CSER_ERR_INVALID, "cser_set_lr: eta must be finite");
+    h->eta = eta;
+    return CSER_OK;
+}
+
 int cser_write_state(cser_handle h, int which, const void *src, size_t bytes, void *stream) {
     if (int rc = check_handle(h)) return rc;
     if (!src) return fail(CSER_ERR_INVALID, "cser_write_state: src is NULL");

@@ -452,6 +452,41 @@ def test_steps_on_a_side_stream_and_kernel_timing_hooks():
     a.close(), c.close()
 
 
+def test_learning_rate_schedule_and_column_reads():
+    d, n, bs = 10_000, 4, 64
+    rng = np.random.default_rng(8)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    opt = b.CSER(d, n, bs, 4, 2, 3, 0.1, 0.9, 6)
+    opt.set_x0(torch.from_numpy(x0).to(DEV))
+    ref = None
+    x_ref = e_ref = m_ref = None
+    lrs = [0.1, 0.1, 0.02, 0.02, 0.004, 0.004]
+    state = None
+    for t, lr in enumerate(lrs, 1):
+        g = rng.standard_normal((n, d)).astype(np.float32)
+        b.cser_set_lr(opt.h, lr)
+        opt.step(torch.from_numpy(g).to(DEV))
+        # oracle with the same schedule: a fresh oracle per learning rate, carrying the state over
+        o = CSEROracle(d, n, bs, 4, 2, 3, lr, 0.9, 6, dtype=np.float32)
+        o.set_x0(x0)
+        if state is not None:
+            o.x, o.e, o.m = state
+        o.t = t - 1
+        o.step(g)
+        state = (o.x, o.e, o.m)
+    assert np.array_equal(opt.state(b.STATE_X).cpu().numpy(), state[0])
+    assert np.array_equal(opt.state(b.STATE_E).cpu().numpy(), state[1])
+    # column window, to device and to host
+    for dev in (DEV, "cpu"):
+        win = torch.empty((n, 300), dtype=torch.float32, device=dev)
+        b.cser_read_columns(opt.h, b.STATE_M, 9_700, 300, win)
+        torch.cuda.synchronize()
+        assert np.array_equal(win.cpu().numpy(), state[2][:, 9_700:])
+    assert b.lib().cser_read_columns(opt.h, b.STATE_X, 9_900, 200, win.data_ptr(), win.numel(), None) == -1
+    assert b.lib().cser_set_lr(opt.h, float("inf")) == -1
+    opt.close()
+
+
 def test_misaligned_gradient_pointer_takes_the_scalar_path():
     d, n = 1024, 4
     rng = np.random.default_rng(3)
