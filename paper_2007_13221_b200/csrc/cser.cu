@@ -1,5 +1,7 @@
-// CSER / M-CSER optimizer step for B200 (sm_100a): GRBS mask kernel, fused step
-// kernel and the C ABI declared in include/cser.h.
+// CSER / M-CSER optimizer step for B200 (sm_100a): host side of the C ABI declared in
+// include/cser.h.  The kernels live in grbs_kernels.cuh (block selection),
+// step_kernels.cuh (streaming and selected-block kernels) and wshard_kernels.cuh
+// (worker-sharded pack / apply).
 //
 // Layout: g, x, e, m are fp32 [n, d] row-major (worker-major).  The step is bound
 // by HBM traffic (about 28 bytes per element and worker against 7 flops), so the
@@ -44,710 +46,9 @@ int fail(int code, const char *fmt, ...) {
                         "%s: %s", #expr, cudaGetErrorString(_e));                         \
     } while (0)
 
-// ------------------------------------------------------------------ Philox4x32-10
-// Salmon et al., SC'11.  Ten rounds; key bumped by the Weyl constants each round.
-__device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t k0, uint32_t k1, uint32_t c0,
-                                                        uint32_t c1, uint32_t c2, uint32_t c3) {
-    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
-    const uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
-#pragma unroll
-    for (int r = 0; r < 10; ++r) {
-        const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
-        const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
-        c0 = hi1 ^ c1 ^ k0;
-        c1 = lo1;
-        c2 = hi0 ^ c3 ^ k1;
-        c3 = lo0;
-        k0 += W0;
-        k1 += W1;
-    }
-    return c0;
-}
-
-// GRBS block select (Definition 2).  Thread idx < B draws the update mask of block
-// idx, thread B <= idx < 2B the reset mask of block idx - B (only on reset steps).
-__global__ void __launch_bounds__(256)
-grbs_mask_kernel(uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r, long long B,
-                 long long block_begin, uint32_t k0, uint32_t k1, uint32_t t_lo, uint32_t t_hi,
-                 uint32_t R_g, uint32_t R_r, int n_masks, uint32_t first_which) {
-    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= B * n_masks) return;
-    const uint32_t second = idx >= B ? 1u : 0u;
-    const long long b = idx - (second ? B : 0);
-    const uint32_t which = first_which + second;
-    const uint32_t R = which ? R_r : R_g;
-    const uint32_t w0 =
-        philox4x32_10_word0(k0, k1, (uint32_t)(block_begin + b), t_lo, t_hi, which);
-    const uint8_t sel = (R != 0 && (unsigned long long)w0 * R < (1ull << 32)) ? 1 : 0;   // R = 0: C = 0
-    (second ? mask_r : mask_g)[b] = sel;
-}
-
-// ------------------------------------------------------------------ exact-count GRBS
-// Definition 2 read literally: exactly k = round(B / R) blocks, those with the k smallest
-// keys (word0, block id).  The k-th smallest key is found in two passes over the B draws
-// with no sorting: a 4096-bin histogram of the top 12 bits of word0 locates the bin that
-// holds it, then the few keys of that bin (about B / 4096) are ranked against each other.
-// Each pass ends in the last CTA to finish (a counter, no waiting), which does the small
-// serial part and re-arms the scratch for the next step.
-constexpr int kExactBins = 4096;
-constexpr int kExactCap = 8192;          // candidate keys kept per mask
-struct ExactScratch {
-    uint32_t hist[2][kExactBins];
-    uint32_t bin[2];                      // bin that holds the k-th smallest key
-    uint32_t k_rem[2];                    // its rank inside that bin (1-based)
-    uint32_t n_cand[2];
-    uint32_t done[2];                     // CTAs finished, one counter per pass
-    unsigned long long thr[2];            // the k-th smallest key
-    unsigned long long cand[2][kExactCap];
-};
-
-__global__ void __launch_bounds__(256)
-grbs_exact_hist_kernel(ExactScratch *__restrict__ X, uint32_t *__restrict__ words, long long B,
-                       uint32_t k0, uint32_t k1, uint32_t t_lo, uint32_t t_hi, uint32_t kg, uint32_t kr,
-                       int n_masks, uint32_t first_which) {
-    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx < B * n_masks) {
-        const uint32_t second = idx >= B ? 1u : 0u;
-        const long long b = idx - (second ? B : 0);
-        const uint32_t which = first_which + second;
-        const uint32_t w = philox4x32_10_word0(k0, k1, (uint32_t)b, t_lo, t_hi, which);
-        words[(size_t)which * B + b] = w;
-        atomicAdd(&X->hist[which][w >> 20], 1u);
-    }
-    __shared__ bool last;
-    __shared__ uint32_t part[256];
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) last = atomicAdd(&X->done[0], 1u) == gridDim.x - 1;
-    __syncthreads();
-    if (!last) return;
-    __threadfence();
-    for (int q = 0; q < n_masks; ++q) {
-        const uint32_t which = first_which + q;
-        const uint32_t k = which ? kr : kg;
-        volatile uint32_t *h = X->hist[which];
-        constexpr int per = kExactBins / 256;
-        uint32_t loc[per], sum = 0;
-#pragma unroll
-        for (int j = 0; j < per; ++j) { loc[j] = h[threadIdx.x * per + j]; sum += loc[j]; }
-        part[threadIdx.x] = sum;
-        __syncthreads();
-        uint32_t before = 0;                        // draws in bins below this thread's bins
-        for (int j = 0; j < (int)threadIdx.x; ++j) before += part[j];
-        if (k > before && k <= before + sum) {      // the k-th smallest lies in one of my bins
-            uint32_t cum = before;
-#pragma unroll
-            for (int j = 0; j < per; ++j) {
-                if (k > cum && k <= cum + loc[j]) {
-                    X->bin[which] = threadIdx.x * per + j;
-                    X->k_rem[which] = k - cum;
-                }
-                cum += loc[j];
-            }
-        }
-        __syncthreads();
-#pragma unroll
-        for (int j = 0; j < per; ++j) h[threadIdx.x * per + j] = 0;   // re-arm for the next step
-        if (threadIdx.x == 0) X->n_cand[which] = 0;
-    }
-    if (threadIdx.x == 0) X->done[0] = 0;
-}
-
-__global__ void __launch_bounds__(256)
-grbs_exact_threshold_kernel(ExactScratch *__restrict__ X, const uint32_t *__restrict__ words, long long B,
-                            int n_masks, uint32_t first_which) {
-    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx < B * n_masks) {
-        const uint32_t second = idx >= B ? 1u : 0u;
-        const long long b = idx - (second ? B : 0);
-        const uint32_t which = first_which + second;
-        const uint32_t w = words[(size_t)which * B + b];
-        if ((w >> 20) == X->bin[which]) {
-            const uint32_t at = atomicAdd(&X->n_cand[which], 1u);
-            if (at < (uint32_t)kExactCap) X->cand[which][at] = ((unsigned long long)w << 32) | (uint32_t)b;
-        }
-    }
-    __shared__ bool last;
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) last = atomicAdd(&X->done[1], 1u) == gridDim.x - 1;
-    __syncthreads();
-    if (!last) return;
-    __threadfence();
-    for (int q = 0; q < n_masks; ++q) {
-        const uint32_t which = first_which + q;
-        const uint32_t m = min(*(volatile uint32_t *)&X->n_cand[which], (uint32_t)kExactCap);
-        const uint32_t want = X->k_rem[which] - 1;   // rank (0-based) of the threshold inside the bin
-        const volatile unsigned long long *c = X->cand[which];
-        for (uint32_t i = threadIdx.x; i < m; i += blockDim.x) {
-            const unsigned long long ki = c[i];
-            uint32_t rank = 0;
-            for (uint32_t j = 0; j < m; ++j) rank += c[j] < ki ? 1u : 0u;
-            if (rank == want) X->thr[which] = ki;   // keys are distinct: exactly one writer
-        }
-    }
-    if (threadIdx.x == 0) X->done[1] = 0;
-}
-
-// Per-step block select: one thread per block.  With `draw` it draws the update mask (and,
-// on a reset step, the reset mask) and stores the flags; without it the flags already in
-// mask_g / mask_r are used (injected masks).  Blocks selected by either mask are appended
-// to `list` (order irrelevant: blocks are independent) with one atomicAdd per warp on
-// *count.  *count_next, the counter the following step will use, is cleared here, so no
-// counter ever needs a separate memset.
-__global__ void __launch_bounds__(256)
-grbs_select_kernel(uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r,
-                   uint32_t *__restrict__ list, uint32_t *count, uint32_t *count_next, long long B,
-                   long long block_begin, uint32_t k0, uint32_t k1, uint32_t t_lo, uint32_t t_hi,
-                   uint32_t R_g, uint32_t R_r, int is_reset, int draw,
-                   const unsigned long long *__restrict__ exact_thr, int exact_g, int exact_r) {
-    const long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (b == 0) *count_next = 0;
-    bool sg = false, sr = false;
-    if (b < B) {
-        if (draw) {
-            const uint32_t gb = (uint32_t)(block_begin + b);
-            // R = 0: the compressor keeps nothing (C = 0).  exact_*: keep the blocks whose key
-            // (word0, block id) is not above the k-th smallest key (exact-count GRBS).
-            if (R_g != 0) {
-                const uint32_t w = philox4x32_10_word0(k0, k1, gb, t_lo, t_hi, 0u);
-                sg = exact_g ? ((((unsigned long long)w << 32) | gb) <= exact_thr[0])
-                             : ((unsigned long long)w * R_g < (1ull << 32));
-            }
-            mask_g[b] = sg ? 1 : 0;
-            if (is_reset) {
-                if (R_r != 0) {
-                    const uint32_t w = philox4x32_10_word0(k0, k1, gb, t_lo, t_hi, 1u);
-                    sr = exact_r ? ((((unsigned long long)w << 32) | gb) <= exact_thr[1])
-                                 : ((unsigned long long)w * R_r < (1ull << 32));
-                }
-                mask_r[b] = sr ? 1 : 0;
-            }
-        } else {
-            sg = mask_g[b] != 0;
-            sr = is_reset ? (mask_r[b] != 0) : false;
-        }
-    }
-    const bool need = sg || sr;
-    const unsigned ballot = __ballot_sync(0xffffffffu, need);
-    if (ballot == 0) return;
-    const unsigned lane = threadIdx.x & 31;
-    const int leader = __ffs(ballot) - 1;
-    unsigned base = 0;
-    if ((int)lane == leader) base = atomicAdd(count, (unsigned)__popc(ballot));
-    base = __shfl_sync(0xffffffffu, base, leader);
-    if (need) list[base + __popc(ballot & ((1u << lane) - 1u))] = (uint32_t)b;
-}
-
-// ------------------------------------------------------------------ fused step
-template <int V>
-struct Pack {
-    float v[V];
-};
-
-template <int V>
-__device__ __forceinline__ Pack<V> ld(const float *p) {
-    Pack<V> r;
-    if constexpr (V == 4) {
-        const float4 t = *reinterpret_cast<const float4 *>(p);
-        r.v[0] = t.x, r.v[1] = t.y, r.v[2] = t.z, r.v[3] = t.w;
-    } else {
-        r.v[0] = *p;
-    }
-    return r;
-}
-
-// gradients are read exactly once: stream them past the caches
-template <int V>
-__device__ __forceinline__ Pack<V> ld_stream(const float *p) {
-    Pack<V> r;
-    if constexpr (V == 4) {
-        const float4 t = __ldcs(reinterpret_cast<const float4 *>(p));
-        r.v[0] = t.x, r.v[1] = t.y, r.v[2] = t.z, r.v[3] = t.w;
-    } else {
-        r.v[0] = __ldcs(p);
-    }
-    return r;
-}
-
-template <int V>
-__device__ __forceinline__ void st(float *p, const Pack<V> &a) {
-    if constexpr (V == 4) {
-        *reinterpret_cast<float4 *>(p) = make_float4(a.v[0], a.v[1], a.v[2], a.v[3]);
-    } else {
-        *p = a.v[0];
-    }
-}
-
-struct StepParams {
-    const float *g;
-    float *x, *e, *m;
-    const uint8_t *mask_g, *mask_r;
-    const uint32_t *list;    // blocks selected by either mask this step
-    const uint32_t *count;   // how many
-    long long d;             // elements per row
-    long long cols_total;    // vector columns per row
-    long long c_begin;       // first vector column handled by this launch
-    long long c_end;         // one past the last
-    unsigned bsv;            // GRBS block size in vector columns
-    unsigned tiles;          // tiles of 256 vector columns in [c_begin, c_end)
-    int n;
-    float eta, beta, n_f;
-};
-
-// Get_p (Appendix A.4) for one pack; updates m in place when MOM.
-template <int V, bool MOM>
-__device__ __forceinline__ Pack<V> get_p(const Pack<V> &g, Pack<V> &m, float eta, float beta) {
-    Pack<V> p;
-#pragma unroll
-    for (int k = 0; k < V; ++k) {
-        if constexpr (MOM) {
-            const float t1 = beta * m.v[k];
-            m.v[k] = t1 + g.v[k];
-            const float t2 = beta * m.v[k];
-            p.v[k] = eta * (t2 + g.v[k]);
-        } else {
-            p.v[k] = eta * g.v[k];
-        }
-    }
-    return p;
-}
-
-constexpr int kStepThreads = 256;   // streaming kernel: one CTA = 256 vector columns of one row
-constexpr int kWalkThreads = 128;   // selected-block kernel
-constexpr int kWalkBatch = 4;       // workers whose loads a walking thread keeps in flight
-#ifndef CSER_DENSE_WALK_FRACTION
-#define CSER_DENSE_WALK_FRACTION 0.3
-#endif
-constexpr double kDenseWalkFraction = CSER_DENSE_WALK_FRACTION;   // expected selected share from which the walk is dense
-
-// Selected blocks (1/R of the data): the update needs the mean over workers, so here one
-// thread owns one vector column of a selected block and walks the worker axis.  Threads
-// are laid over the concatenation of the listed blocks, so CTAs are full whatever the
-// block size.  Each pass issues the loads of kWalkBatch workers before it consumes any of
-// them (the in-place stores would otherwise keep the compiler from hoisting the next
-// worker's loads), and sums in ascending worker order starting from worker 0's value.
-// This kernel has its own register budget; the streaming kernel stays at 32 registers.
-// DENSE = false: threads are laid over the listed blocks (few blocks selected).  DENSE =
-// true: one thread per column of the whole range, returning at once if no mask selects its
-// block; used when a large share of the blocks is selected, where walking the columns in
-// their natural order is worth more than the idle threads cost.
-template <int V, bool MOM, bool RESET, bool ERR, bool DENSE>
-__global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepParams P) {
-    constexpr int U = kWalkBatch;
-    const unsigned long long total =
-        DENSE ? (unsigned long long)(P.c_end - P.c_begin) : (unsigned long long)(*P.count) * P.bsv;
-    const long long d = P.d;
-    const int n = P.n;
-    const float eta = P.eta, beta = P.beta;
-    for (unsigned long long f = (unsigned long long)blockIdx.x * kWalkThreads + threadIdx.x; f < total;
-         f += (unsigned long long)gridDim.x * kWalkThreads) {
-        long long c;
-        unsigned blk;
-        if constexpr (DENSE) {
-            c = P.c_begin + (long long)f;
-            blk = (P.c_end <= 0xffffffffll) ? (uint32_t)c / P.bsv : (unsigned)((unsigned long long)c / P.bsv);
-        } else {
-            const unsigned long long entry =
-                (total <= 0xffffffffull) ? (unsigned long long)((uint32_t)f / P.bsv) : f / P.bsv;
-            blk = P.list[entry];
-            c = (long long)blk * P.bsv + (long long)(f - entry * P.bsv);
-            if (c >= P.cols_total || c < P.c_begin || c >= P.c_end) continue;
-        }
-        const bool sg = P.mask_g[blk] != 0;
-        const bool sr = RESET ? (P.mask_r[blk] != 0) : false;
-        if constexpr (DENSE) {
-            if (!sg && !sr) continue;
-        }
-        const float *__restrict__ g = P.g + c * V;
-        float *__restrict__ x = P.x + c * V;
-        float *__restrict__ e = ERR ? P.e + c * V : nullptr;
-        float *__restrict__ m = MOM ? P.m + c * V : nullptr;
-        // With an error array: sum over workers of e_{t-1/2}.  Without one (implementation
-        // II): sum over workers of x_{t-1/2}.  Reset-selected blocks only.
-        Pack<V> sum_r;
-#pragma unroll
-        for (int k = 0; k < V; ++k) sum_r.v[k] = 0.f;
-
-        if (sg) {
-            // Update-selected block: r = 0, p' = mean_k p_k.  Pass A forms the mean and updates m.
-            Pack<V> sum_p;
-#pragma unroll
-            for (int k = 0; k < V; ++k) sum_p.v[k] = 0.f;
-            for (int i0 = 0; i0 < n; i0 += U) {
-                Pack<V> gv[U], mv[U];
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    if (i0 + u < n) {
-                        const long long o = (long long)(i0 + u) * d;
-                        gv[u] = ld_stream<V>(g + o);
-                        if constexpr (MOM) mv[u] = ld<V>(m + o);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    if (i0 + u < n) {
-                        const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], eta, beta);
-                        if constexpr (MOM) st<V>(m + (long long)(i0 + u) * d, mv[u]);
-#pragma unroll
-                        for (int k = 0; k < V; ++k)
-                            sum_p.v[k] = (i0 + u == 0) ? p.v[k] : sum_p.v[k] + p.v[k];
-                    }
-                }
-            }
-            Pack<V> pbar;
-#pragma unroll
-            for (int k = 0; k < V; ++k) pbar.v[k] = sum_p.v[k] / P.n_f;
-            // Pass B: x_i -= p-bar; e untouched.  If the block is reset-selected too: with an
-            // error array store (x_i - p-bar) - e_i, zero e and gather sum_k e_k; without one
-            // gather sum_k (x_k - p-bar) and store nothing yet.
-            for (int i0 = 0; i0 < n; i0 += U) {
-                Pack<V> xv[U], ev[U];
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    if (i0 + u < n) {
-                        const long long o = (long long)(i0 + u) * d;
-                        xv[u] = ld<V>(x + o);
-                        if constexpr (ERR) {
-                            if (sr) ev[u] = ld<V>(e + o);
-                        }
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    if (i0 + u < n) {
-                        const long long o = (long long)(i0 + u) * d;
-#pragma unroll
-                        for (int k = 0; k < V; ++k) xv[u].v[k] = xv[u].v[k] - pbar.v[k];
-                        if (sr) {
-                            if constexpr (ERR) {
-                                Pack<V> z;
-#pragma unroll
-                                for (int k = 0; k < V; ++k) {
-                                    sum_r.v[k] = (i0 + u == 0) ? ev[u].v[k] : sum_r.v[k] + ev[u].v[k];
-                                    xv[u].v[k] = xv[u].v[k] - ev[u].v[k];
-                                    z.v[k] = 0.f;
-                                }
-                                st<V>(e + o, z);
-                                st<V>(x + o, xv[u]);
-                            } else {
-#pragma unroll
-                                for (int k = 0; k < V; ++k)
-                                    sum_r.v[k] = (i0 + u == 0) ? xv[u].v[k] : sum_r.v[k] + xv[u].v[k];
-                            }
-                        } else {
-                            st<V>(x + o, xv[u]);
-                        }
-                    }
-                }
-            }
-        } else {
-            // Selected by the reset mask only: take the residual step (x_{t-1/2} = x - p,
-            // e_{t-1/2} = e - p).  With an error array store x_{t-1/2} - e_{t-1/2}, zero e and
-            // gather sum_k e_{k,t-1/2}; without one gather sum_k x_{k,t-1/2}.
-            constexpr int U2 = 2;
-            for (int i0 = 0; i0 < n; i0 += U2) {
-                Pack<V> gv[U2], mv[U2], xv[U2], ev[U2];
-#pragma unroll
-                for (int u = 0; u < U2; ++u) {
-                    if (i0 + u < n) {
-                        const long long o = (long long)(i0 + u) * d;
-                        gv[u] = ld_stream<V>(g + o);
-                        if constexpr (MOM) mv[u] = ld<V>(m + o);
-                        xv[u] = ld<V>(x + o);
-                        if constexpr (ERR) ev[u] = ld<V>(e + o);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < U2; ++u) {
-                    if (i0 + u < n) {
-                        const long long o = (long long)(i0 + u) * d;
-                        const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], eta, beta);
-                        if constexpr (MOM) st<V>(m + o, mv[u]);
-                        if constexpr (ERR) {
-                            Pack<V> z;
-#pragma unroll
-                            for (int k = 0; k < V; ++k) {
-                                const float xh = xv[u].v[k] - p.v[k];
-                                const float eh = ev[u].v[k] - p.v[k];
-                                sum_r.v[k] = (i0 + u == 0) ? eh : sum_r.v[k] + eh;
-                                xv[u].v[k] = xh - eh;
-                                z.v[k] = 0.f;
-                            }
-                            st<V>(x + o, xv[u]);
-                            st<V>(e + o, z);
-                        } else {
-#pragma unroll
-                            for (int k = 0; k < V; ++k) {
-                                const float xh = xv[u].v[k] - p.v[k];
-                                sum_r.v[k] = (i0 + u == 0) ? xh : sum_r.v[k] + xh;
-                            }
-                        }
-                    }
-                }
-            }
-        }
-
-        if (sr) {
-            Pack<V> rbar;
-#pragma unroll
-            for (int k = 0; k < V; ++k) rbar.v[k] = sum_r.v[k] / P.n_f;
-            if constexpr (ERR) {
-                // Error reset (Algorithm 2 lines 11-12):
-                // x_i = (x_{i,t-1/2} - e_{i,t-1/2}) + mean_k e_{k,t-1/2}.
-                for (int i0 = 0; i0 < n; i0 += U) {
-                    Pack<V> xv[U];
-#pragma unroll
-                    for (int u = 0; u < U; ++u)
-                        if (i0 + u < n) xv[u] = ld<V>(x + (long long)(i0 + u) * d);
-#pragma unroll
-                    for (int u = 0; u < U; ++u) {
-                        if (i0 + u < n) {
-#pragma unroll
-                            for (int k = 0; k < V; ++k) xv[u].v[k] = xv[u].v[k] + rbar.v[k];
-                            st<V>(x + (long long)(i0 + u) * d, xv[u]);
-                        }
-                    }
-                }
-            } else {
-                // Implementation II (Appendix A.4): x_i = mean_k x_{k,t-1/2} for every worker.
-                for (int i = 0; i < n; ++i) st<V>(x + (long long)i * d, rbar);
-            }
-        }
-    }
-}
-
-// Unselected blocks (all but 1/R of the data), purely elementwise.  1-D grid: CTA
-// i * tiles + tile streams tile `tile` of worker i, so consecutive CTAs walk one row after
-// the other, contiguously.  Thread t owns vector column c = c_begin + 256 * tile + t and
-// leaves it alone if a mask selects its block.
-template <int V, bool MOM, bool RESET, bool ERR>
-__global__ void __launch_bounds__(kStepThreads, 8) cser_stream_kernel(const StepParams P) {
-    const unsigned row = blockIdx.x / P.tiles;
-    const unsigned tile = blockIdx.x - row * P.tiles;
-    const long long c = P.c_begin + (long long)tile * kStepThreads + threadIdx.x;
-    if (c >= P.c_end) return;
-    const long long b = (P.c_end <= 0xffffffffll) ? (long long)((uint32_t)c / P.bsv)
-                                                  : (long long)((unsigned long long)c / P.bsv);
-    if (P.mask_g[b] != 0) return;
-    if (RESET && P.mask_r[b] != 0) return;
-    // C(p) = 0, so p' = r = p (Algorithm 3 lines 4-8): x_i -= p_i, e_i -= p_i (no e array in
-    // implementation II).
-    const long long o = (long long)row * P.d + c * V;
-    const Pack<V> gv = ld_stream<V>(P.g + o);
-    Pack<V> mv;
-    if constexpr (MOM) mv = ld<V>(P.m + o);
-    Pack<V> xv = ld<V>(P.x + o);
-    Pack<V> ev;
-    if constexpr (ERR) ev = ld<V>(P.e + o);
-    const Pack<V> p = get_p<V, MOM>(gv, mv, P.eta, P.beta);
-#pragma unroll
-    for (int k = 0; k < V; ++k) {
-        xv.v[k] = xv.v[k] - p.v[k];
-        if constexpr (ERR) ev.v[k] = ev.v[k] - p.v[k];
-    }
-    if constexpr (MOM) st<V>(P.m + o, mv);
-    st<V>(P.x + o, xv);
-    if constexpr (ERR) st<V>(P.e + o, ev);
-}
-
-// ------------------------------------------------------------------ worker-sharded step
-// Several GPUs each hold some of the workers (all d columns).  The mean of Algorithm 3 line 7
-// then needs one all-reduce per step.  GRBS makes the compressed vectors directly summable
-// (Section 3.3): every rank selects the same blocks, so each rank packs the sum over its own
-// workers of the selected blocks into a dense message, the messages are summed across ranks,
-// and each rank applies sum / n_total.  The message holds the update-selected blocks in
-// ascending block order and, on a reset step, the reset-selected blocks after them.
-
-// Exclusive scan of the two masks in block order (one CTA): pos_*[b] = selected blocks below b,
-// olist_* = the selected blocks in ascending order.
-__global__ void __launch_bounds__(1024)
-ordered_lists_kernel(const uint8_t *__restrict__ mask_g, const uint8_t *__restrict__ mask_r, long long B,
-                     int is_reset, uint32_t *__restrict__ pos_g, uint32_t *__restrict__ pos_r,
-                     uint32_t *__restrict__ olist_g, uint32_t *__restrict__ olist_r) {
-    __shared__ uint32_t part[2][1024];
-    const long long chunk = (B + blockDim.x - 1) / blockDim.x;
-    const long long b0 = min(B, (long long)threadIdx.x * chunk), b1 = min(B, b0 + chunk);
-    uint32_t cg = 0, cr = 0;
-    for (long long b = b0; b < b1; ++b) {
-        cg += mask_g[b] != 0;
-        if (is_reset) cr += mask_r[b] != 0;
-    }
-    part[0][threadIdx.x] = cg, part[1][threadIdx.x] = cr;
-    __syncthreads();
-    uint32_t og = 0, orr = 0;
-    for (int j = 0; j < (int)threadIdx.x; ++j) og += part[0][j], orr += part[1][j];
-    for (long long b = b0; b < b1; ++b) {
-        pos_g[b] = og;
-        if (mask_g[b]) olist_g[og++] = (uint32_t)b;
-        if (is_reset) {
-            pos_r[b] = orr;
-            if (mask_r[b]) olist_r[orr++] = (uint32_t)b;
-        }
-    }
-}
-
-struct ShardParams {
-    const float *g;
-    float *x, *e, *m;
-    float *msg;                       // [k_g * bs | k_r * bs] floats
-    const uint8_t *mask_g, *mask_r;
-    const uint32_t *pos_g, *olist_g, *olist_r;
-    long long d, cols_total;
-    unsigned bsv, k_g, k_r;
-    int n;                            // local workers
-    float eta, beta, n_total_f;
-};
-
-// Pack: thread f owns vector column (f % bsv) of message block (f / bsv).
-template <int V, bool MOM, bool RESET>
-__global__ void __launch_bounds__(kWalkThreads) wshard_pack_kernel(const ShardParams P) {
-    constexpr int U = kWalkBatch;
-    const unsigned long long total = (unsigned long long)(P.k_g + (RESET ? P.k_r : 0u)) * P.bsv;
-    const long long d = P.d;
-    const int n = P.n;
-    for (unsigned long long f = (unsigned long long)blockIdx.x * kWalkThreads + threadIdx.x; f < total;
-         f += (unsigned long long)gridDim.x * kWalkThreads) {
-        const unsigned entry = (unsigned)(f / P.bsv);
-        const unsigned col = (unsigned)(f - (unsigned long long)entry * P.bsv);
-        const bool r_section = entry >= P.k_g;
-        const unsigned blk = r_section ? P.olist_r[entry - P.k_g] : P.olist_g[entry];
-        const long long c = (long long)blk * P.bsv + col;
-        Pack<V> sum;
-#pragma unroll
-        for (int q = 0; q < V; ++q) sum.v[q] = 0.f;
-        if (c < P.cols_total) {
-            const float *__restrict__ g = P.g + c * V;
-            float *__restrict__ x = P.x + c * V;
-            float *__restrict__ e = P.e + c * V;
-            float *__restrict__ m = MOM ? P.m + c * V : nullptr;
-            if (!r_section) {
-                // update-selected block: sum of the local workers' p, ascending; m updated
-                for (int i0 = 0; i0 < n; i0 += U) {
-                    Pack<V> gv[U], mv[U];
-#pragma unroll
-                    for (int u = 0; u < U; ++u) {
-                        if (i0 + u < n) {
-                            const long long o = (long long)(i0 + u) * d;
-                            gv[u] = ld_stream<V>(g + o);
-                            if constexpr (MOM) mv[u] = ld<V>(m + o);
-                        }
-                    }
-#pragma unroll
-                    for (int u = 0; u < U; ++u) {
-                        if (i0 + u < n) {
-                            const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], P.eta, P.beta);
-                            if constexpr (MOM) st<V>(m + (long long)(i0 + u) * d, mv[u]);
-#pragma unroll
-                            for (int q = 0; q < V; ++q) sum.v[q] = (i0 + u == 0) ? p.v[q] : sum.v[q] + p.v[q];
-                        }
-                    }
-                }
-            } else if (P.mask_g[blk] != 0) {
-                // reset-selected and update-selected: e is unchanged by this step; sum the local e
-                for (int i = 0; i < n; ++i) {
-                    const Pack<V> ev = ld<V>(e + (long long)i * d);
-#pragma unroll
-                    for (int q = 0; q < V; ++q) sum.v[q] = (i == 0) ? ev.v[q] : sum.v[q] + ev.v[q];
-                }
-            } else {
-                // reset-selected only: residual step, store x_{t-1/2} - e_{t-1/2}, zero e, sum e_{t-1/2}
-                for (int i = 0; i < n; ++i) {
-                    const long long o = (long long)i * d;
-                    const Pack<V> gv = ld_stream<V>(g + o);
-                    Pack<V> mv, xv = ld<V>(x + o);
-                    const Pack<V> ev = ld<V>(e + o);
-                    if constexpr (MOM) mv = ld<V>(m + o);
-                    const Pack<V> p = get_p<V, MOM>(gv, mv, P.eta, P.beta);
-                    if constexpr (MOM) st<V>(m + o, mv);
-                    Pack<V> z;
-#pragma unroll
-                    for (int q = 0; q < V; ++q) {
-                        const float xh = xv.v[q] - p.v[q];
-                        const float eh = ev.v[q] - p.v[q];
-                        sum.v[q] = (i == 0) ? eh : sum.v[q] + eh;
-                        xv.v[q] = xh - eh;
-                        z.v[q] = 0.f;
-                    }
-                    st<V>(x + o, xv);
-                    st<V>(e + o, z);
-                }
-            }
-        }
-        st<V>(P.msg + ((size_t)entry * P.bsv + col) * V, sum);   // columns past the end of the vector: zeros
-    }
-}
-
-// Apply the summed message: thread f owns one vector column of one message block.
-template <int V, bool RESET>
-__global__ void __launch_bounds__(kWalkThreads) wshard_apply_kernel(const ShardParams P) {
-    const unsigned long long total = (unsigned long long)(P.k_g + (RESET ? P.k_r : 0u)) * P.bsv;
-    const long long d = P.d;
-    const int n = P.n;
-    for (unsigned long long f = (unsigned long long)blockIdx.x * kWalkThreads + threadIdx.x; f < total;
-         f += (unsigned long long)gridDim.x * kWalkThreads) {
-        const unsigned entry = (unsigned)(f / P.bsv);
-        const unsigned col = (unsigned)(f - (unsigned long long)entry * P.bsv);
-        const bool r_section = entry >= P.k_g;
-        const unsigned blk = r_section ? P.olist_r[entry - P.k_g] : P.olist_g[entry];
-        const long long c = (long long)blk * P.bsv + col;
-        if (c >= P.cols_total) continue;
-        float *__restrict__ x = P.x + c * V;
-        float *__restrict__ e = P.e + c * V;
-        const Pack<V> sv = ld<V>(P.msg + ((size_t)entry * P.bsv + col) * V);
-        Pack<V> mean;
-#pragma unroll
-        for (int q = 0; q < V; ++q) mean.v[q] = sv.v[q] / P.n_total_f;
-        if (!r_section) {
-            if (RESET && P.mask_r[blk] != 0) continue;   // its reset-section thread does both updates
-            for (int i = 0; i < n; ++i) {                // x_i -= mean_k p_k
-                Pack<V> xv = ld<V>(x + (long long)i * d);
-#pragma unroll
-                for (int q = 0; q < V; ++q) xv.v[q] = xv.v[q] - mean.v[q];
-                st<V>(x + (long long)i * d, xv);
-            }
-        } else if (P.mask_g[blk] != 0) {
-            // both masks: x_i = ((x_i - p-bar) - e_i) + e-bar, e_i = 0
-            const Pack<V> sp = ld<V>(P.msg + ((size_t)P.pos_g[blk] * P.bsv + col) * V);
-            for (int i = 0; i < n; ++i) {
-                const long long o = (long long)i * d;
-                Pack<V> xv = ld<V>(x + o);
-                const Pack<V> ev = ld<V>(e + o);
-                Pack<V> z;
-#pragma unroll
-                for (int q = 0; q < V; ++q) {
-                    const float pbar = sp.v[q] / P.n_total_f;
-                    xv.v[q] = ((xv.v[q] - pbar) - ev.v[q]) + mean.v[q];
-                    z.v[q] = 0.f;
-                }
-                st<V>(x + o, xv);
-                st<V>(e + o, z);
-            }
-        } else {
-            for (int i = 0; i < n; ++i) {                // x_i = (x_{t-1/2} - e_{t-1/2}) + e-bar
-                Pack<V> xv = ld<V>(x + (long long)i * d);
-#pragma unroll
-                for (int q = 0; q < V; ++q) xv.v[q] = xv.v[q] + mean.v[q];
-                st<V>(x + (long long)i * d, xv);
-            }
-        }
-    }
-}
-
-// x_i <- x0 for all workers; e, m <- 0
-__global__ void __launch_bounds__(256)
-broadcast_x0_kernel(const float *__restrict__ x0, float *__restrict__ x, float *__restrict__ e,
-                    float *__restrict__ m, long long d, int n) {
-    const long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= d) return;
-    const float v = x0[j];
-    for (int i = 0; i < n; ++i) {
-        const long long o = (long long)i * d + j;
-        x[o] = v;
-        if (e) e[o] = 0.f;
-        if (m) m[o] = 0.f;
-    }
-}
+#include "grbs_kernels.cuh"
+#include "step_kernels.cuh"
+#include "wshard_kernels.cuh"
 
 }  // namespace
 

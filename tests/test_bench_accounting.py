@@ -1,0 +1,33 @@
+"""The roofline numerator: bytes a step must move, per element and worker, for the five workloads.
+
+g is read (4 B), x read and written (8 B), m read and written when there is momentum (8 B), e read and
+written only where it is touched: everywhere but the update-selected blocks on a plain step (fraction
+1 - 1/R1), and on a reset step also on the reset-selected ones (1 - (1/R1)(1 - 1/R2)).
+"""
+import pytest
+
+import bench
+from paper_2007_13221_b200 import synth
+
+
+@pytest.mark.parametrize("cfg,per_elt,gb_per_step", [(1, 18.125, 0.1520), (2, 27.751, 7.9365), (3, 27.969, 11.4370),
+                                                     (4, 27.992, 5.7232), (5, 27.875, 74.7373)])
+def test_algorithmic_bytes_per_workload(cfg, per_elt, gb_per_step):
+    w = synth.CONFIGS[cfg]
+    mean = bench.mean_algorithmic_bytes(w, 1, w.H)           # one reset in H steps
+    assert abs(mean / (w.n_workers * w.d) - per_elt) < 5e-4
+    assert abs(mean / 1e9 - gb_per_step) < 5e-4 * gb_per_step + 1e-4
+
+
+def test_variants_change_the_count_as_stated():
+    w = synth.CONFIGS[2]
+    assert bench.algorithmic_bytes(w, 1.0) == w.n_workers * w.d * 28
+    bench.NO_ERROR_ARRAY = True
+    try:
+        assert bench.algorithmic_bytes(w, 1.0) == w.n_workers * w.d * 20
+    finally:
+        bench.NO_ERROR_ARRAY = False
+    from dataclasses import replace
+    assert bench.expected_e_fraction(replace(w, R1=0), False) == 1.0      # C2 = 0: e touched everywhere
+    assert bench.expected_e_fraction(replace(w, R1=1, R2=1), True) == 1.0
+    assert bench.expected_e_fraction(replace(w, R1=1), False) == 0.0      # everything synchronized: e idle
