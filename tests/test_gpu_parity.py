@@ -507,6 +507,52 @@ def test_misaligned_gradient_pointer_takes_the_scalar_path():
     opt.close()
 
 
+# ------------------------------------------------------------------ randomized differential test
+def test_random_shapes_parameters_and_flags_against_the_float32_oracle():
+    """400 random problems (shape, ratios, reset interval, momentum, flags, injected masks now and
+    then, host-gradient entry now and then): the state must equal the float32 oracle exactly."""
+    rng = np.random.default_rng(20240607)
+    for case in range(400):
+        n = int(rng.choice([1, 2, 3, 4, 5, 8, 9, 16, 17]))
+        bs = int(rng.choice([1, 3, 4, 8, 12, 16, 60, 64, 100, 128, 256]))
+        d = int(rng.integers(1, 40)) * bs + int(rng.integers(0, bs)) if rng.random() < 0.7 else int(rng.integers(1, 3000))
+        R1 = int(rng.choice([0, 1, 2, 3, 4, 7, 32]))
+        R2 = int(rng.choice([1, 2, 3, 4, 16]))
+        H = int(rng.integers(1, 5))
+        beta = float(rng.choice([0.0, 0.5, 0.9]))
+        eta = float(rng.choice([0.1, 0.01, 1.0]))
+        impl2 = rng.random() < 0.3
+        exact = rng.random() < 0.3
+        seed = int(rng.integers(0, 2**62))
+        flags = (b.FLAG_NO_ERROR_ARRAY if impl2 else 0) | (b.FLAG_EXACT_COUNT if exact else 0)
+        opt = b.CSER(d, n, bs, R1, R2, H, eta, beta, seed, flags=flags)
+        ref = (CSERImpl2Oracle if impl2 else CSEROracle)(d, n, bs, R1, R2, H, eta, beta, seed, dtype=np.float32,
+                                                         exact_count=exact)
+        x0 = rng.standard_normal(d).astype(np.float32)
+        opt.set_x0(torch.from_numpy(x0).to(DEV) if rng.random() < 0.5 else torch.from_numpy(x0))
+        ref.set_x0(x0)
+        B = n_blocks(d, bs)
+        label = (case, d, n, bs, R1, R2, H, beta, flags)
+        for t in range(1, int(rng.integers(3, 9))):
+            g = rng.standard_normal((n, d)).astype(np.float32)
+            if rng.random() < 0.15:                    # injected masks for this step
+                mg = rng.integers(0, 2, B).astype(np.uint8)
+                mr = rng.integers(0, 2, B).astype(np.uint8)
+                opt.inject_masks(torch.from_numpy(mg).to(DEV), torch.from_numpy(mr).to(DEV))
+                ref.inject_masks(mg, mr)
+            if rng.random() < 0.2:
+                opt.step_host(torch.from_numpy(g).pin_memory())
+            else:
+                opt.step(torch.from_numpy(g).to(DEV))
+            ref.step(g)
+            assert np.array_equal(opt.state(b.STATE_MASK_G).cpu().numpy(), ref.mask_g), label + (t, "mask")
+        names = ((b.STATE_X, "x"),) + (() if impl2 else ((b.STATE_E, "e"),)) + (((b.STATE_M, "m"),) if beta else ())
+        for which, name in names:
+            got, want = opt.state(which).cpu().numpy(), getattr(ref, name)
+            assert np.array_equal(got, want), label + (name, int((got != want).sum()))
+        opt.close()
+
+
 # ------------------------------------------------------------------ boundary behaviour
 def test_host_gradient_entry_point_equals_device_entry_point():
     w = synth.CONFIGS[2].scaled(d=3_000_000 + 4, steps=10)
