@@ -77,7 +77,15 @@ __device__ __forceinline__ Pack<V> get_p(const Pack<V> &g, Pack<V> &m, float eta
 
 constexpr int kStepThreads = 256;   // streaming kernel: one CTA = 256 vector columns of one row
 constexpr int kWalkThreads = 128;   // selected-block kernel
-constexpr int kWalkBatch = 4;       // workers whose loads a walking thread keeps in flight
+constexpr int kWalkBatch = 4;       // workers whose loads a walking thread keeps in flight (worker-sharded pack)
+// Batch sizes of the selected-block kernel.  Measured on B200: 2, 4 and 8 are within 2 % of each
+// other on every workload (more loads in flight per thread cost registers, hence occupancy).
+#ifndef CSER_WALK_UA
+#define CSER_WALK_UA(mom) 4
+#define CSER_WALK_UB(reset_err) 4
+#define CSER_WALK_UF 4
+#define CSER_WALK_UR(mom) 2
+#endif
 #ifndef CSER_DENSE_WALK_FRACTION
 #define CSER_DENSE_WALK_FRACTION 0.3
 #endif
@@ -96,7 +104,10 @@ constexpr double kDenseWalkFraction = CSER_DENSE_WALK_FRACTION;   // expected se
 // their natural order is worth more than the idle threads cost.
 template <int V, bool MOM, bool RESET, bool ERR, bool DENSE>
 __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepParams P) {
-    constexpr int U = kWalkBatch;
+    // workers whose loads are in flight together: fewer arrays per worker allow more workers
+    constexpr int UA = CSER_WALK_UA(MOM);                      // pass A: g (+ m)
+    constexpr int UB = CSER_WALK_UB(RESET && ERR);             // pass B: x (+ e on reset steps)
+    constexpr int UF = CSER_WALK_UF;                           // last pass: x only
     const unsigned long long total =
         DENSE ? (unsigned long long)(P.c_end - P.c_begin) : (unsigned long long)(*P.count) * P.bsv;
     const long long d = P.d;
@@ -136,10 +147,10 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
             Pack<V> sum_p;
 #pragma unroll
             for (int k = 0; k < V; ++k) sum_p.v[k] = 0.f;
-            for (int i0 = 0; i0 < n; i0 += U) {
-                Pack<V> gv[U], mv[U];
+            for (int i0 = 0; i0 < n; i0 += UA) {
+                Pack<V> gv[UA], mv[UA];
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
+                for (int u = 0; u < UA; ++u) {
                     if (i0 + u < n) {
                         const long long o = (long long)(i0 + u) * d;
                         gv[u] = ld_stream<V>(g + o);
@@ -147,7 +158,7 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
                     }
                 }
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
+                for (int u = 0; u < UA; ++u) {
                     if (i0 + u < n) {
                         const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], eta, beta);
                         if constexpr (MOM) st<V>(m + (long long)(i0 + u) * d, mv[u]);
@@ -163,10 +174,10 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
             // Pass B: x_i -= p-bar; e untouched.  If the block is reset-selected too: with an
             // error array store (x_i - p-bar) - e_i, zero e and gather sum_k e_k; without one
             // gather sum_k (x_k - p-bar) and store nothing yet.
-            for (int i0 = 0; i0 < n; i0 += U) {
-                Pack<V> xv[U], ev[U];
+            for (int i0 = 0; i0 < n; i0 += UB) {
+                Pack<V> xv[UB], ev[UB];
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
+                for (int u = 0; u < UB; ++u) {
                     if (i0 + u < n) {
                         const long long o = (long long)(i0 + u) * d;
                         xv[u] = ld<V>(x + o);
@@ -176,7 +187,7 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
                     }
                 }
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
+                for (int u = 0; u < UB; ++u) {
                     if (i0 + u < n) {
                         const long long o = (long long)(i0 + u) * d;
 #pragma unroll
@@ -207,7 +218,7 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
             // Selected by the reset mask only: take the residual step (x_{t-1/2} = x - p,
             // e_{t-1/2} = e - p).  With an error array store x_{t-1/2} - e_{t-1/2}, zero e and
             // gather sum_k e_{k,t-1/2}; without one gather sum_k x_{k,t-1/2}.
-            constexpr int U2 = 2;
+            constexpr int U2 = CSER_WALK_UR(MOM);             // g, x, e (+ m)
             for (int i0 = 0; i0 < n; i0 += U2) {
                 Pack<V> gv[U2], mv[U2], xv[U2], ev[U2];
 #pragma unroll
@@ -257,13 +268,13 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
             if constexpr (ERR) {
                 // Error reset (Algorithm 2 lines 11-12):
                 // x_i = (x_{i,t-1/2} - e_{i,t-1/2}) + mean_k e_{k,t-1/2}.
-                for (int i0 = 0; i0 < n; i0 += U) {
-                    Pack<V> xv[U];
+                for (int i0 = 0; i0 < n; i0 += UF) {
+                    Pack<V> xv[UF];
 #pragma unroll
-                    for (int u = 0; u < U; ++u)
+                    for (int u = 0; u < UF; ++u)
                         if (i0 + u < n) xv[u] = ld<V>(x + (long long)(i0 + u) * d);
 #pragma unroll
-                    for (int u = 0; u < U; ++u) {
+                    for (int u = 0; u < UF; ++u) {
                         if (i0 + u < n) {
 #pragma unroll
                             for (int k = 0; k < V; ++k) xv[u].v[k] = xv[u].v[k] + rbar.v[k];
