@@ -89,11 +89,14 @@ def _check(rc, what):
 
 
 def _stream(stream=None):
-    return ctypes.c_void_p((stream or torch.cuda.current_stream()).cuda_stream)
+    """Raw cudaStream_t of `stream`, or of torch's current stream on the current device."""
+    if stream is not None:
+        return stream.cuda_stream
+    return torch._C._cuda_getCurrentRawStream(torch.cuda.current_device())
 
 
 def _ptr(t):
-    return ctypes.c_void_p(t.data_ptr())
+    return t.data_ptr()
 
 
 FLAG_NO_ERROR_ARRAY = 1
@@ -118,7 +121,9 @@ def cser_set_x0(h, x0, stream=None):
 
 def cser_step(h, grad, stream=None):
     assert grad.dtype == torch.float32 and grad.is_contiguous() and grad.is_cuda
-    _check(lib().cser_step(h, _ptr(grad), _stream(stream)), "cser_step")
+    rc = _lib.cser_step(h, grad.data_ptr(), _stream(stream))       # hot path: nothing else per call
+    if rc:
+        _check(rc, "cser_step")
 
 
 def cser_step_host(h, grad_host, stream=None):

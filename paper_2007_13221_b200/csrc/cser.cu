@@ -91,6 +91,7 @@ struct cser_ctx {
     // auxiliary stream they run side by side (fork after the select kernel, join after both).
     cudaStream_t aux = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    const float *last_grad_checked = nullptr;        // last gradient pointer verified to be device memory
     float *x0_stage = nullptr;                       // [d] staging for a host x0
     bool masks_injected = false;
     bool vec4 = false;                               // 128-bit path usable for the state arrays
@@ -457,7 +458,10 @@ int cser_set_x0(cser_handle h, const float *x0, void *stream) {
 
 int cser_step(cser_handle h, const float *grad, void *stream) {
     if (int rc = check_handle(h)) return rc;
-    if (int rc = check_device_ptr(grad, "cser_step: grad")) return rc;
+    if (!grad || grad != h->last_grad_checked) {   // the pointer query costs a microsecond: once per buffer
+        if (int rc = check_device_ptr(grad, "cser_step: grad")) return rc;
+        h->last_grad_checked = grad;
+    }
     if ((uintptr_t)grad % 4 != 0) return fail(CSER_ERR_INVALID, "cser_step: grad is not 4-byte aligned");
     if (h->n_total > 0) return fail(CSER_ERR_INVALID, "cser_step: worker-sharded handle; use cser_wshard_pack/apply");
     cudaStream_t s = (cudaStream_t)stream;
