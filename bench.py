@@ -33,6 +33,7 @@ NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2_wrn40x8_n8_R32_H8": 1.7983e9 * 35_748_708 
 
 NO_ERROR_ARRAY = False   # --impl2: implementation II of Appendix A.4 (no e array)
 EXACT_COUNT = False      # --exact-count: every mask selects exactly round(B/R) blocks
+L2_RESIDENT = False      # ask the library to keep a small state in L2 (CSER_FLAG_L2_RESIDENT)
 
 
 def algorithmic_bytes(w, frac_e_touched):
@@ -255,7 +256,8 @@ def run_workload(w, K, W, dev, rank, world, ring_n=0, with_e2e=True, flush_l2=Fa
     # each rank owns one slab of the workload's size, with global block ids
     opt = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
                  block_begin=0 if EXACT_COUNT else rank * w.n_blocks,
-                 flags=(b.FLAG_NO_ERROR_ARRAY if NO_ERROR_ARRAY else 0) | (b.FLAG_EXACT_COUNT if EXACT_COUNT else 0))
+                 flags=(b.FLAG_NO_ERROR_ARRAY if NO_ERROR_ARRAY else 0) | (b.FLAG_EXACT_COUNT if EXACT_COUNT else 0)
+                 | (b.FLAG_L2_RESIDENT if L2_RESIDENT else 0))
     opt.set_x0(synth.x0(w, dev))
     g_bytes = w.n_workers * w.d * 4
     ring_n = ring_n or max(2, min(4, int(6e9 // g_bytes)))
@@ -481,6 +483,15 @@ def main():
         guarded(w.name + " implementation II (no error array, 20 B per element-worker)", lambda: variant("impl2"))
         for c in (1, 3, 4, 5):
             guarded(synth.CONFIGS[c].name, lambda c=c: other_workload(c))
+
+        def l2_resident():
+            global L2_RESIDENT
+            try:
+                L2_RESIDENT = True
+                return other_workload(1)
+            finally:
+                L2_RESIDENT = False
+        guarded(synth.CONFIGS[1].name + " with the state kept in L2 (CSER_FLAG_L2_RESIDENT)", l2_resident)
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

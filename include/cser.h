@@ -123,6 +123,15 @@ cser_handle cser_create_slab(int64_t d, int32_t n_workers, int32_t block_size,
  *       2^22 blocks.
  */
 #define CSER_FLAG_EXACT_COUNT 2u
+/*
+ *   CSER_FLAG_L2_RESIDENT  if x, e and m together fit the part of the GPU's L2 cache that can
+ *       be set aside for persisting lines (about 79 MB on B200), keep them there: the step
+ *       kernels are launched with an access-policy window over the state, so only the
+ *       gradients stream from HBM.  The set-aside is a limit of the whole CUDA context: it
+ *       takes that much L2 away from every other kernel of the process until the handle is
+ *       destroyed, which is why it is opt-in.  Ignored when the state does not fit.
+ */
+#define CSER_FLAG_L2_RESIDENT 4u
 cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size,
                            uint32_t R1, uint32_t R2, int32_t H,
                            float eta, float beta, uint64_t seed, int64_t block_begin,

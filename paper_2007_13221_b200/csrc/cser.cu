@@ -59,7 +59,13 @@ struct cser_ctx {
     uint32_t R1 = 1, R2 = 1;
     float eta = 0.f, beta = 0.f;
     uint64_t seed = 0, t = 0;
-    float *x = nullptr, *e = nullptr, *m = nullptr;
+    float *x = nullptr, *e = nullptr, *m = nullptr;   // carved out of one allocation, state_base
+    void *state_base = nullptr;
+    size_t state_bytes = 0;
+    // A state that fits the part of L2 that can be set aside for persisting lines is kept there:
+    // the step kernels are launched with an access-policy window over the state.
+    bool l2_persist = false;
+    size_t l2_limit_before = 0;
     // Masks and list of the current step (aliases of one of the two buffer sets below).
     uint8_t *mask_g = nullptr, *mask_r = nullptr;
     uint32_t *sel_list = nullptr;                    // [B] blocks selected this step
@@ -232,13 +238,28 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     }
     const bool dense = frac >= kDenseWalkFraction;
     if (dense) wgrid = wmax;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeAccessPolicyWindow;
+    attr[0].val.accessPolicyWindow.base_ptr = h->state_base;
+    attr[0].val.accessPolicyWindow.num_bytes = h->state_bytes;
+    attr[0].val.accessPolicyWindow.hitRatio = 1.0f;
+    attr[0].val.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
+    attr[0].val.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
+    auto launch = [&](void (*kernel)(const StepParams), unsigned g, unsigned threads, cudaStream_t st) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(g), cfg.blockDim = dim3(threads), cfg.dynamicSmemBytes = 0, cfg.stream = st;
+        cfg.attrs = attr, cfg.numAttrs = h->l2_persist ? 1 : 0;
+        return cudaLaunchKernelEx(&cfg, kernel, Q);
+    };
+    cudaError_t lerr = cudaSuccess;
 #define CSER_LAUNCH_PAIR(MOM_, RESET_, ERR_)                                                            \
     do {                                                                                                \
         if (dense)                                                                                      \
-            cser_selected_kernel<V, MOM_, RESET_, ERR_, true><<<(unsigned)wgrid, kWalkThreads, 0, ws>>>(Q);  \
+            lerr = launch(cser_selected_kernel<V, MOM_, RESET_, ERR_, true>, (unsigned)wgrid, kWalkThreads, ws); \
         else                                                                                            \
-            cser_selected_kernel<V, MOM_, RESET_, ERR_, false><<<(unsigned)wgrid, kWalkThreads, 0, ws>>>(Q); \
-        if (stream_any) cser_stream_kernel<V, MOM_, RESET_, ERR_><<<grid, kStepThreads, 0, s>>>(Q);     \
+            lerr = launch(cser_selected_kernel<V, MOM_, RESET_, ERR_, false>, (unsigned)wgrid, kWalkThreads, ws); \
+        if (stream_any && lerr == cudaSuccess)                                                          \
+            lerr = launch(cser_stream_kernel<V, MOM_, RESET_, ERR_>, grid, kStepThreads, s);            \
     } while (0)
 #define CSER_LAUNCH_ERR(MOM_, RESET_)                                                                   \
     do {                                                                                                \
@@ -255,6 +276,7 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
 #undef CSER_LAUNCH_ERR
 #undef CSER_LAUNCH_PAIR
     h->launches += stream_any ? 2 : 1;
+    CU_TRY(lerr);
     CU_TRY(cudaGetLastError());
     if (fork) {
         int rc = CSER_OK;
@@ -338,7 +360,7 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
         fail(CSER_ERR_INVALID, "cser_create: d, n_workers, block_size, R2, H must be positive");
         return nullptr;
     }
-    if (flags & ~(uint32_t)(CSER_FLAG_NO_ERROR_ARRAY | CSER_FLAG_EXACT_COUNT)) {
+    if (flags & ~(uint32_t)(CSER_FLAG_NO_ERROR_ARRAY | CSER_FLAG_EXACT_COUNT | CSER_FLAG_L2_RESIDENT)) {
         fail(CSER_ERR_INVALID, "cser_create: unknown flags 0x%x", flags);
         return nullptr;
     }
@@ -366,10 +388,18 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
     h->vec4 = (d % 4 == 0) && (block_size % 4 == 0);
     const size_t bytes = state_elems(h) * sizeof(float);
     cudaError_t er = cudaGetDevice(&h->device);
-    if (er == cudaSuccess) er = cudaMalloc(&h->x, bytes);
-    const bool with_e = !(flags & CSER_FLAG_NO_ERROR_ARRAY);
-    if (er == cudaSuccess && with_e) er = cudaMalloc(&h->e, bytes);
-    if (er == cudaSuccess && beta != 0.f) er = cudaMalloc(&h->m, bytes);
+    // x, e, m in one allocation (each array starts on a 256-byte boundary)
+    const bool with_e_ = !(flags & CSER_FLAG_NO_ERROR_ARRAY);
+    const size_t arr_bytes = (bytes + 255) / 256 * 256;
+    const int n_arrays = 1 + (with_e_ ? 1 : 0) + (beta != 0.f ? 1 : 0);
+    h->state_bytes = arr_bytes * n_arrays;
+    if (er == cudaSuccess) er = cudaMalloc(&h->state_base, h->state_bytes);
+    if (er == cudaSuccess) {
+        char *p = static_cast<char *>(h->state_base);
+        h->x = reinterpret_cast<float *>(p), p += arr_bytes;
+        if (with_e_) h->e = reinterpret_cast<float *>(p), p += arr_bytes;
+        if (beta != 0.f) h->m = reinterpret_cast<float *>(p);
+    }
     for (auto &sb : h->sb) {
         if (er == cudaSuccess) er = cudaMalloc(&sb.mask_g, (size_t)B);
         if (er == cudaSuccess) er = cudaMalloc(&sb.mask_r, (size_t)B);
@@ -377,9 +407,22 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
         if (er == cudaSuccess) er = cudaMemset(sb.mask_g, 0, (size_t)B);
         if (er == cudaSuccess) er = cudaMemset(sb.mask_r, 0, (size_t)B);
     }
-    if (er == cudaSuccess) er = cudaMemset(h->x, 0, bytes);
-    if (er == cudaSuccess && h->e) er = cudaMemset(h->e, 0, bytes);
-    if (er == cudaSuccess && h->m) er = cudaMemset(h->m, 0, bytes);
+    if (er == cudaSuccess) er = cudaMemset(h->state_base, 0, h->state_bytes);
+    if (er == cudaSuccess && (flags & CSER_FLAG_L2_RESIDENT)) {
+        // Keep a small state resident in L2 (set-aside persisting lines); larger ones stream.
+        int max_persist = 0, max_window = 0;
+        cudaDeviceGetAttribute(&max_persist, cudaDevAttrMaxPersistingL2CacheSize, h->device);
+        cudaDeviceGetAttribute(&max_window, cudaDevAttrMaxAccessPolicyWindowSize, h->device);
+        if (h->state_bytes <= (size_t)max_persist && h->state_bytes <= (size_t)max_window) {
+            size_t cur_limit = 0;
+            if (cudaDeviceGetLimit(&cur_limit, cudaLimitPersistingL2CacheSize) == cudaSuccess) {
+                h->l2_limit_before = cur_limit;
+                const size_t want = cur_limit > h->state_bytes ? cur_limit : h->state_bytes;
+                h->l2_persist = cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want) == cudaSuccess;
+            }
+            cudaGetLastError();
+        }
+    }
     h->exact = (flags & CSER_FLAG_EXACT_COUNT) != 0;
     if (er == cudaSuccess && h->exact) er = cudaMalloc(&h->exact_scratch, sizeof(ExactScratch));
     if (er == cudaSuccess && h->exact) er = cudaMemset(h->exact_scratch, 0, sizeof(ExactScratch));
@@ -419,7 +462,12 @@ cser_handle cser_create(int64_t d, int32_t n_workers, int32_t block_size, uint32
 
 void cser_destroy(cser_handle h) {
     if (!h) return;
-    cudaFree(h->x), cudaFree(h->e), cudaFree(h->m);
+    if (h->l2_persist) {
+        cudaCtxResetPersistingL2Cache();
+        cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, h->l2_limit_before);
+        cudaGetLastError();
+    }
+    cudaFree(h->state_base);
     for (auto &sb : h->sb) cudaFree(sb.mask_g), cudaFree(sb.mask_r), cudaFree(sb.list);
     cudaFree(h->x0_stage), cudaFree(h->g_stage);
     cudaFree(h->sel_count), cudaFree(h->exact_scratch), cudaFree(h->exact_words);

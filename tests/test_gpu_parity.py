@@ -487,6 +487,22 @@ def test_learning_rate_schedule_and_column_reads():
     opt.close()
 
 
+def test_l2_resident_state_gives_the_same_results():
+    w = synth.CONFIGS[1].scaled(d=300_000, steps=9)          # 9.6 MB of state: fits the L2 set-aside
+    a = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, 3)
+    c = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, 3, flags=b.FLAG_L2_RESIDENT)
+    big = b.CSER(30_000_000, 8, 256, 4, 4, 4, 0.1, 0.0, 3, flags=b.FLAG_L2_RESIDENT)   # 1.9 GB: flag ignored
+    x0 = synth.x0(w, DEV)
+    a.set_x0(x0), c.set_x0(x0)
+    for t in range(1, w.steps + 1):
+        g = synth.gradients(w, t, DEV)
+        a.step(g), c.step(g)
+    big.step(torch.zeros((8, 30_000_000), device=DEV))
+    for which in (b.STATE_X, b.STATE_E):
+        assert torch.equal(a.state(which), c.state(which))
+    a.close(), c.close(), big.close()
+
+
 def test_misaligned_gradient_pointer_takes_the_scalar_path():
     d, n = 1024, 4
     rng = np.random.default_rng(3)
