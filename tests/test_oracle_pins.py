@@ -482,3 +482,28 @@ def test_exact_count_mode_keeps_the_invariants():
         assert int(o.mask_g.sum()) == exact_count(o.B, 4)
         assert np.allclose(o.x.mean(0), xbar, atol=1e-12)
         assert np.abs((o.x - o.e) - (o.x - o.e)[0]).max() < 1e-12
+
+
+# --------------------------------------------------------------------------- Lemma 3 (error after a reset is bounded)
+def test_error_after_reset_stays_below_the_bound_of_lemma_3():
+    """E||e_{i,t}||^2 <= (1 - d2)(1 - d1) eta^2 H^2 V2 / (1 - sqrt(1 - d1))^2 at every t with t mod H = 0,
+    with d2 = 1/R1 (update compressor), d1 = 1/R2 (reset compressor) and V2 >= E||g||^2."""
+    n, d, bs, R1, R2, H, eta, T = 4, 512, 8, 4, 2, 4, 0.1, 40
+    d1, d2 = 1.0 / R2, 1.0 / R1
+    sq = {t: [] for t in range(H, T + 1, H)}
+    g_sq = []
+    for seed in range(30):
+        rng = np.random.default_rng(1000 + seed)
+        o = CSEROracle(d, n, bs, R1, R2, H, eta, 0.0, seed)
+        o.set_x0(rng.standard_normal(d))
+        for t in range(1, T + 1):
+            g = rng.standard_normal((n, d))
+            g_sq.append((g**2).sum(1).mean())
+            o.step(g)
+            if t % H == 0:
+                sq[t].append((o.e**2).sum(1).mean())
+    V2 = float(np.mean(g_sq))
+    bound = (1 - d2) * (1 - d1) * float(np.float32(eta)) ** 2 * H**2 * V2 / (1 - np.sqrt(1 - d1)) ** 2
+    worst = max(float(np.mean(v)) for v in sq.values())
+    assert 0 < worst <= bound
+    assert worst > 1e-3 * bound            # the bound is loose but not vacuous for this setting
