@@ -153,6 +153,8 @@ int cser_set_x0(cser_handle h, const float *x0, void *stream);
  * Increments t, then enqueues the step kernels (and, beside them, the GRBS select kernel of
  * the following iteration, whose masks depend only on seed and t; the first step, and a step
  * after cser_set_x0, cser_write_state(T) or cser_debug_set_masks, runs its own first).
+ * The iteration number is passed to the kernels by value, so the launches of one call
+ * belong to that iteration only: a stream capture of cser_step must not be replayed.
  */
 int cser_step(cser_handle h, const float *grad, void *stream);
 
