@@ -375,6 +375,44 @@ def run_worker_sharded(w, K, W, dev):
     return out
 
 
+def run_graph_replay(w, K, dev):
+    """One replayable step captured in a CUDA graph (torch is the plumbing for the capture), replayed K times."""
+    import torch
+    from paper_2007_13221_b200 import binding as b, synth
+    opt = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed)
+    opt.set_x0(synth.x0(w, dev))
+    g = synth.gradients(w, 1, dev)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        b.cser_replay_begin(opt.h)
+        for _ in range(3):
+            b.cser_step_replayable(opt.h, g)
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side, capture_error_mode="thread_local"):
+        b.cser_step_replayable(opt.h, g)
+    for _ in range(5):
+        graph.replay()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(K):
+        graph.replay()
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / K
+    t_end = opt.t
+    b.cser_replay_end(opt.h)
+    alg = mean_algorithmic_bytes(w, 1, w.H)
+    out = {"steps_per_s": 1e3 / ms, "ms_per_step": ms, "steps": K, "iterations_done": t_end,
+           "hbm_gbs_step": alg / (ms * 1e-3) / 1e9, "hbm_frac_of_8TBs": alg / (ms * 1e-3) / 1e9 / PEAK_NOMINAL_GBS}
+    opt.close()
+    del g, graph
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -492,6 +530,9 @@ def main():
             finally:
                 L2_RESIDENT = False
         guarded(synth.CONFIGS[1].name + " with the state kept in L2 (CSER_FLAG_L2_RESIDENT)", l2_resident)
+        guarded(synth.CONFIGS[1].name + " step captured in a CUDA graph and replayed",
+                lambda: run_graph_replay(synth.CONFIGS[1], 2000, dev))
+        guarded(w.name + " step captured in a CUDA graph and replayed", lambda: run_graph_replay(w, 100, dev))
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

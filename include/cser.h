@@ -159,6 +159,25 @@ int cser_set_x0(cser_handle h, const float *x0, void *stream);
 int cser_step(cser_handle h, const float *grad, void *stream);
 
 /*
+ * Replayable steps, for callers that capture their training iteration in a CUDA graph.
+ * Between cser_replay_begin and cser_replay_end the step counter lives in device memory and
+ * is advanced by the step itself, so the launches enqueued by one call of
+ * cser_step_replayable perform "the next iteration", whichever that is: they may be captured
+ * once (stream capture of the call on `stream`) and replayed any number of times; every
+ * replay is one more iteration of Algorithm 2 / 4 on whatever the gradient buffer then holds.
+ * The call may also be used without capture.  Results are the same as cser_step's.
+ * cser_replay_begin copies the host step counter to the device (and synchronizes `stream`);
+ * cser_replay_end synchronizes `stream` and reads it back.  In between, cser_step,
+ * cser_step_host, cser_set_x0, cser_write_state and cser_debug_set_masks are refused;
+ * cser_read_state works (the step counter is read from the device).  Not available with
+ * exact-count masks or worker-sharded handles.  grad must be the same pointer at replay time
+ * as at capture time (a captured launch carries its arguments).
+ */
+int cser_replay_begin(cser_handle h, void *stream);
+int cser_step_replayable(cser_handle h, const float *grad, void *stream);
+int cser_replay_end(cser_handle h, void *stream);
+
+/*
  * The same iteration with the gradients in HOST memory (pinned memory gives
  * asynchronous copies): the library copies them, slab by slab, into a device
  * staging buffer it owns (allocated on the first such call, n*d*4 bytes) and runs

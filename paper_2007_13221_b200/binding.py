@@ -55,6 +55,11 @@ def lib():
     L.cser_step_host.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p]
     L.cser_read_state.argtypes = [c.c_void_p, c.c_int, c.c_void_p, c.c_size_t, c.c_void_p]
     L.cser_write_state.argtypes = [c.c_void_p, c.c_int, c.c_void_p, c.c_size_t, c.c_void_p]
+    for name in ("cser_replay_begin", "cser_replay_end"):
+        getattr(L, name).restype = c.c_int
+        getattr(L, name).argtypes = [c.c_void_p, c.c_void_p]
+    L.cser_step_replayable.restype = c.c_int
+    L.cser_step_replayable.argtypes = [c.c_void_p, c.c_void_p, c.c_void_p]
     L.cser_read_columns.restype = c.c_int
     L.cser_read_columns.argtypes = [c.c_void_p, c.c_int, c.c_int64, c.c_int64, c.c_void_p, c.c_size_t, c.c_void_p]
     L.cser_set_lr.restype = c.c_int
@@ -135,6 +140,19 @@ def cser_step_host(h, grad_host, stream=None):
 def cser_read_state(h, which, dst, stream=None):
     _check(lib().cser_read_state(h, which, _ptr(dst), dst.numel() * dst.element_size(), _stream(stream)),
            "cser_read_state")
+
+
+def cser_replay_begin(h, stream=None):
+    _check(lib().cser_replay_begin(h, _stream(stream)), "cser_replay_begin")
+
+
+def cser_step_replayable(h, grad, stream=None):
+    assert grad.dtype == torch.float32 and grad.is_contiguous() and grad.is_cuda
+    _check(lib().cser_step_replayable(h, grad.data_ptr(), _stream(stream)), "cser_step_replayable")
+
+
+def cser_replay_end(h, stream=None):
+    _check(lib().cser_replay_end(h, _stream(stream)), "cser_replay_end")
 
 
 def cser_read_columns(h, which, col_begin, col_count, dst, stream=None):

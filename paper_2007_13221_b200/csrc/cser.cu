@@ -84,6 +84,9 @@ struct cser_ctx {
     uint64_t pre_t = 0;
     const uint32_t *pre_count = nullptr;
     bool walk_all = false;                           // masks were injected: no estimate of the selected count
+    // replayable steps (cser_replay_begin .. cser_replay_end): the iteration lives on the device
+    StepCtl *ctl = nullptr;
+    bool replay = false;
     // worker-sharded mode (cser_create_wshard): n = local workers, n_total = all ranks' workers
     int n_total = 0;
     uint32_t *pos_g = nullptr, *pos_r = nullptr, *olist_g = nullptr, *olist_r = nullptr;
@@ -193,6 +196,7 @@ int select_for_iteration(cser_ctx *h, bool is_reset, cudaStream_t s) {
 
 template <int V>
 int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t s, bool use_aux) {
+    // (is_reset is a by-value copy: replay mode overrides it below)
     const long long cols = P.c_end - P.c_begin;
     if (cols <= 0) return CSER_OK;
     const long long tiles = (cols + kStepThreads - 1) / kStepThreads;
@@ -200,6 +204,8 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     if (grid_ll > 0x7fffffffll) return fail(CSER_ERR_INVALID, "n_workers * d too large for one launch");
     StepParams Q = P;
     Q.tiles = (unsigned)tiles;
+    Q.ctl = h->replay ? h->ctl : nullptr;
+    if (h->replay) is_reset = true;   // the reset variants decide on the device whether this step resets
     const unsigned grid = (unsigned)grid_ll;
     // Grid of the selected-block kernel: the count lives on the device, so size the grid for
     // the expected number of selected columns in this launch's range plus slack; the kernel
@@ -216,6 +222,7 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     const bool stream_any = h->walk_all || h->R1 != 1;
     cudaStream_t ws = s;
     const bool fork = use_aux && h->aux != nullptr && stream_any;
+    const bool prefetch = !h->replay && h->n_buf == 2;
     if (fork) {
         CU_TRY(cudaEventRecord(h->ev_fork, s));
         CU_TRY(cudaStreamWaitEvent(h->aux, h->ev_fork, 0));
@@ -280,7 +287,7 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     CU_TRY(cudaGetLastError());
     if (fork) {
         int rc = CSER_OK;
-        if (h->n_buf == 2) {
+        if (prefetch) {
             // next iteration's select kernel, off the critical path
             const uint64_t t_next = h->t + 1;
             rc = launch_select(h, h->cur ^ 1, t_next, (t_next % (uint64_t)h->H) == 0, true, h->aux,
@@ -302,7 +309,7 @@ int launch_step(cser_ctx *h, const float *grad, long long col0, long long col1, 
     P.g = grad, P.x = h->x, P.e = h->e, P.m = h->m;
     P.mask_g = h->mask_g, P.mask_r = h->mask_r;
     P.list = h->sel_list, P.count = h->cur_count;
-    P.tiles = 0;
+    P.tiles = 0, P.ctl = nullptr;
     P.d = h->d, P.n = h->n;
     P.eta = h->eta, P.beta = h->beta, P.n_f = (float)h->n;
     const bool v4 = h->vec4 && ((uintptr_t)grad % 16 == 0) && (col0 % 4 == 0) &&
@@ -427,6 +434,8 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
     if (er == cudaSuccess && h->exact) er = cudaMalloc(&h->exact_scratch, sizeof(ExactScratch));
     if (er == cudaSuccess && h->exact) er = cudaMemset(h->exact_scratch, 0, sizeof(ExactScratch));
     if (er == cudaSuccess && h->exact) er = cudaMalloc(&h->exact_words, 2 * (size_t)B * sizeof(uint32_t));
+    if (er == cudaSuccess) er = cudaMalloc(&h->ctl, sizeof(StepCtl));
+    if (er == cudaSuccess) er = cudaMemset(h->ctl, 0, sizeof(StepCtl));
     if (er == cudaSuccess) er = cudaMalloc(&h->sel_count, 3 * sizeof(uint32_t));
     if (er == cudaSuccess) er = cudaMemset(h->sel_count, 0, 3 * sizeof(uint32_t));
     if (er == cudaSuccess) activate_selection(h, 0, h->sel_count, true);
@@ -470,7 +479,7 @@ void cser_destroy(cser_handle h) {
     cudaFree(h->state_base);
     for (auto &sb : h->sb) cudaFree(sb.mask_g), cudaFree(sb.mask_r), cudaFree(sb.list);
     cudaFree(h->x0_stage), cudaFree(h->g_stage);
-    cudaFree(h->sel_count), cudaFree(h->exact_scratch), cudaFree(h->exact_words);
+    cudaFree(h->sel_count), cudaFree(h->exact_scratch), cudaFree(h->exact_words), cudaFree(h->ctl);
     cudaFree(h->pos_g), cudaFree(h->pos_r), cudaFree(h->olist_g), cudaFree(h->olist_r);
     for (auto &ev : h->ev) if (ev) cudaEventDestroy(ev);
     for (auto &ev : h->h_ev) if (ev) cudaEventDestroy(ev);
@@ -484,6 +493,7 @@ void cser_destroy(cser_handle h) {
 int cser_set_x0(cser_handle h, const float *x0, void *stream) {
     if (int rc = check_handle(h)) return rc;
     if (!x0) return fail(CSER_ERR_INVALID, "cser_set_x0: x0 is NULL");
+    if (h->replay) return fail(CSER_ERR_INVALID, "cser_set_x0: call cser_replay_end first");
     cudaStream_t s = (cudaStream_t)stream;
     cudaPointerAttributes a;
     cudaError_t er = cudaPointerGetAttributes(&a, x0);
@@ -512,6 +522,7 @@ int cser_step(cser_handle h, const float *grad, void *stream) {
     }
     if ((uintptr_t)grad % 4 != 0) return fail(CSER_ERR_INVALID, "cser_step: grad is not 4-byte aligned");
     if (h->n_total > 0) return fail(CSER_ERR_INVALID, "cser_step: worker-sharded handle; use cser_wshard_pack/apply");
+    if (h->replay) return fail(CSER_ERR_INVALID, "cser_step: between cser_replay_begin and cser_replay_end use cser_step_replayable");
     cudaStream_t s = (cudaStream_t)stream;
     const bool is_reset = begin_iteration(h);
     if (h->timing) CU_TRY(cudaEventRecord(h->ev[0], s));
@@ -529,6 +540,7 @@ int cser_step_host(cser_handle h, const float *grad_host, void *stream) {
     if (int rc = check_handle(h)) return rc;
     if (!grad_host) return fail(CSER_ERR_INVALID, "cser_step_host: grad_host is NULL");
     if (h->n_total > 0) return fail(CSER_ERR_INVALID, "cser_step_host: worker-sharded handle");
+    if (h->replay) return fail(CSER_ERR_INVALID, "cser_step_host: call cser_replay_end first");
     cudaStream_t s = (cudaStream_t)stream;
     if (!h->g_stage) {
         CU_TRY(cudaMalloc(&h->g_stage, state_elems(h) * sizeof(float)));
@@ -590,6 +602,11 @@ int cser_read_state(cser_handle h, int which, void *dst, size_t dst_bytes, void 
     if (dst_bytes < bytes)
         return fail(CSER_ERR_TOO_SMALL, "cser_read_state: need %zu bytes, got %zu", bytes, dst_bytes);
     if (which == CSER_STATE_T) {
+        if (h->replay) {   // the counter lives on the device while steps are replayable
+            CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+            CU_TRY(cudaMemcpy(dst, &h->ctl->t, sizeof(uint64_t), cudaMemcpyDefault));
+            return CSER_OK;
+        }
         CU_TRY(cudaMemcpy(dst, &h->t, sizeof(uint64_t), cudaMemcpyDefault));
         return CSER_OK;
     }
@@ -627,6 +644,7 @@ int cser_set_lr(cser_handle h, float eta) {
 int cser_write_state(cser_handle h, int which, const void *src, size_t bytes, void *stream) {
     if (int rc = check_handle(h)) return rc;
     if (!src) return fail(CSER_ERR_INVALID, "cser_write_state: src is NULL");
+    if (h->replay) return fail(CSER_ERR_INVALID, "cser_write_state: call cser_replay_end first");
     if (which == CSER_STATE_MASK_G || which == CSER_STATE_MASK_R)
         return fail(CSER_ERR_INVALID, "masks cannot be written; use cser_debug_set_masks");
     void *dst;
@@ -646,6 +664,7 @@ int cser_write_state(cser_handle h, int which, const void *src, size_t bytes, vo
 int cser_debug_set_masks(cser_handle h, const uint8_t *g_mask, const uint8_t *r_mask, void *stream) {
     if (int rc = check_handle(h)) return rc;
     if (!g_mask) return fail(CSER_ERR_INVALID, "cser_debug_set_masks: g_mask is NULL");
+    if (h->replay) return fail(CSER_ERR_INVALID, "cser_debug_set_masks: call cser_replay_end first");
     const bool next_is_reset = ((h->t + 1) % (uint64_t)h->H) == 0;
     if (next_is_reset && !r_mask)
         return fail(CSER_ERR_INVALID, "cser_debug_set_masks: next step resets, r_mask is NULL");
@@ -783,6 +802,54 @@ int cser_wshard_apply(cser_handle h, const float *msg, void *stream) {
                       : launch_wshard<1>(h, P, h->wshard_reset, false, (cudaStream_t)stream);
     if (rc) return rc;
     h->wshard_open = false;
+    return CSER_OK;
+}
+
+int cser_replay_begin(cser_handle h, void *stream) {
+    if (int rc = check_handle(h)) return rc;
+    if (h->replay) return fail(CSER_ERR_INVALID, "cser_replay_begin: already begun");
+    if (h->exact || h->n_total > 0 || h->masks_injected)
+        return fail(CSER_ERR_INVALID,
+                    "cser_replay_begin: not available with exact-count masks, worker sharding or injected masks");
+    StepCtl c = {};
+    c.t = h->t;
+    CU_TRY(cudaMemcpyAsync(h->ctl, &c, sizeof(c), cudaMemcpyHostToDevice, (cudaStream_t)stream));
+    CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));   // c is on this function's stack
+    h->pre_valid = false;
+    activate_selection(h, 0, nullptr, true);
+    h->replay = true;
+    return CSER_OK;
+}
+
+int cser_step_replayable(cser_handle h, const float *grad, void *stream) {
+    if (int rc = check_handle(h)) return rc;
+    if (!h->replay) return fail(CSER_ERR_INVALID, "cser_step_replayable: call cser_replay_begin first");
+    if (!grad || grad != h->last_grad_checked) {
+        if (int rc = check_device_ptr(grad, "cser_step_replayable: grad")) return rc;
+        h->last_grad_checked = grad;
+    }
+    if ((uintptr_t)grad % 4 != 0) return fail(CSER_ERR_INVALID, "cser_step_replayable: grad is not 4-byte aligned");
+    cudaStream_t s = (cudaStream_t)stream;
+    const unsigned grid = (unsigned)((h->B + 255) / 256);
+    grbs_select_replay_kernel<<<grid, 256, 0, s>>>(h->ctl, h->sb[0].mask_g, h->sb[0].mask_r, h->sb[0].list, h->B,
+                                                   h->block_begin, (uint32_t)(h->seed & 0xffffffffu),
+                                                   (uint32_t)(h->seed >> 32), h->R1, h->R2, (uint32_t)h->H);
+    h->launches++;
+    CU_TRY(cudaGetLastError());
+    h->walk_all = false;
+    return launch_step(h, grad, 0, h->d, true, s, true);
+}
+
+int cser_replay_end(cser_handle h, void *stream) {
+    if (int rc = check_handle(h)) return rc;
+    if (!h->replay) return fail(CSER_ERR_INVALID, "cser_replay_end: not begun");
+    CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    StepCtl c = {};
+    CU_TRY(cudaMemcpy(&c, h->ctl, sizeof(c), cudaMemcpyDeviceToHost));
+    h->t = c.t;
+    h->replay = false;
+    h->pre_valid = false;
+    if (c.reset) h->last_mask_r = h->sb[0].mask_r;
     return CSER_OK;
 }
 

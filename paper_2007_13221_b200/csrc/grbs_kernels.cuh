@@ -178,3 +178,60 @@ grbs_select_kernel(uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r,
     if (need) list[base + __popc(ballot & ((1u << lane) - 1u))] = (uint32_t)b;
 }
 
+
+// ------------------------------------------------------------------ replayable steps
+// For a step that is captured once in a CUDA graph and replayed, the iteration number cannot
+// be a launch argument.  It lives in this device-side block instead: the select kernel of a
+// step works on iteration ctl->t + 1 and its last CTA to finish publishes it (t, whether it
+// resets), after which the step kernels of the same step read it.  The two list counters are
+// used alternately by the parity of t.
+struct StepCtl {
+    unsigned long long t;      // last iteration whose select kernel has completed
+    uint32_t reset;            // that iteration is a reset step
+    uint32_t done;             // CTAs of the running select kernel that have finished
+    uint32_t count[2];         // selected-block counters, indexed by t & 1
+};
+
+__global__ void __launch_bounds__(256)
+grbs_select_replay_kernel(StepCtl *ctl, uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r,
+                          uint32_t *__restrict__ list, long long B, long long block_begin, uint32_t k0,
+                          uint32_t k1, uint32_t R_g, uint32_t R_r, uint32_t H) {
+    // Every thread reads t before any CTA can publish the new one: publishing needs all CTAs done.
+    const unsigned long long t = *(volatile unsigned long long *)&ctl->t + 1ull;
+    const bool is_reset = (t % H) == 0;
+    const uint32_t t_lo = (uint32_t)(t & 0xffffffffu), t_hi = (uint32_t)(t >> 32);
+    uint32_t *count = &ctl->count[t & 1];
+    const long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (b == 0) ctl->count[(t + 1) & 1] = 0;     // the previous step's kernels have finished with it
+    bool sg = false, sr = false;
+    if (b < B) {
+        const uint32_t gb = (uint32_t)(block_begin + b);
+        if (R_g != 0)
+            sg = (unsigned long long)philox4x32_10_word0(k0, k1, gb, t_lo, t_hi, 0u) * R_g < (1ull << 32);
+        mask_g[b] = sg ? 1 : 0;
+        if (is_reset) {
+            sr = (unsigned long long)philox4x32_10_word0(k0, k1, gb, t_lo, t_hi, 1u) * R_r < (1ull << 32);
+            mask_r[b] = sr ? 1 : 0;
+        }
+    }
+    const bool need = sg || sr;
+    const unsigned ballot = __ballot_sync(0xffffffffu, need);
+    if (ballot != 0) {
+        const unsigned lane = threadIdx.x & 31;
+        const int leader = __ffs(ballot) - 1;
+        unsigned base = 0;
+        if ((int)lane == leader) base = atomicAdd(count, (unsigned)__popc(ballot));
+        base = __shfl_sync(0xffffffffu, base, leader);
+        if (need) list[base + __popc(ballot & ((1u << lane) - 1u))] = (uint32_t)b;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(&ctl->done, 1u) == gridDim.x - 1) {   // last CTA: everything above is visible
+            ctl->reset = is_reset ? 1u : 0u;
+            ctl->done = 0;
+            __threadfence();
+            *(volatile unsigned long long *)&ctl->t = t;
+        }
+    }
+}

@@ -47,6 +47,7 @@ struct StepParams {
     const uint8_t *mask_g, *mask_r;
     const uint32_t *list;    // blocks selected by either mask this step
     const uint32_t *count;   // how many
+    const StepCtl *ctl;      // replayable steps: iteration, reset flag and counters on the device (else NULL)
     long long d;             // elements per row
     long long cols_total;    // vector columns per row
     long long c_begin;       // first vector column handled by this launch
@@ -108,8 +109,10 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
     constexpr int UA = CSER_WALK_UA(MOM);                      // pass A: g (+ m)
     constexpr int UB = CSER_WALK_UB(RESET && ERR);             // pass B: x (+ e on reset steps)
     constexpr int UF = CSER_WALK_UF;                           // last pass: x only
+    const uint32_t n_listed = DENSE ? 0u : (P.ctl ? P.ctl->count[P.ctl->t & 1] : *P.count);
+    const bool reset_on = RESET && (P.ctl ? P.ctl->reset != 0 : true);
     const unsigned long long total =
-        DENSE ? (unsigned long long)(P.c_end - P.c_begin) : (unsigned long long)(*P.count) * P.bsv;
+        DENSE ? (unsigned long long)(P.c_end - P.c_begin) : (unsigned long long)n_listed * P.bsv;
     const long long d = P.d;
     const int n = P.n;
     const float eta = P.eta, beta = P.beta;
@@ -128,7 +131,7 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
             if (c >= P.cols_total || c < P.c_begin || c >= P.c_end) continue;
         }
         const bool sg = P.mask_g[blk] != 0;
-        const bool sr = RESET ? (P.mask_r[blk] != 0) : false;
+        const bool sr = reset_on ? (P.mask_r[blk] != 0) : false;
         if constexpr (DENSE) {
             if (!sg && !sr) continue;
         }
@@ -303,7 +306,7 @@ __global__ void __launch_bounds__(kStepThreads, 8) cser_stream_kernel(const Step
     const long long b = (P.c_end <= 0xffffffffll) ? (long long)((uint32_t)c / P.bsv)
                                                   : (long long)((unsigned long long)c / P.bsv);
     if (P.mask_g[b] != 0) return;
-    if (RESET && P.mask_r[b] != 0) return;
+    if (RESET && P.mask_r[b] != 0 && (P.ctl == nullptr || P.ctl->reset != 0)) return;
     // C(p) = 0, so p' = r = p (Algorithm 3 lines 4-8): x_i -= p_i, e_i -= p_i (no e array in
     // implementation II).
     const long long o = (long long)row * P.d + c * V;

@@ -523,6 +523,76 @@ def test_misaligned_gradient_pointer_takes_the_scalar_path():
     opt.close()
 
 
+# ------------------------------------------------------------------ replayable steps and CUDA graphs
+@pytest.mark.parametrize("d,n,bs,R1,R2,H,beta,flags", [
+    (4096 + 40, 8, 256, 4, 2, 3, 0.9, 0), (1001, 3, 7, 2, 3, 2, 0.0, 0), (50_000, 16, 512, 8, 4, 1, 0.9, 0),
+    (20_000, 4, 64, 1, 2, 4, 0.9, 0), (30_000, 8, 128, 0, 2, 2, 0.0, 0), (30_000, 8, 128, 4, 4, 2, 0.9, 1)])
+def test_replayable_steps_equal_ordinary_steps_and_the_oracle(d, n, bs, R1, R2, H, beta, flags):
+    """cser_step, then replayable steps (not captured), then cser_step again: one trajectory."""
+    rng = np.random.default_rng(77)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    impl2 = bool(flags & b.FLAG_NO_ERROR_ARRAY)
+    opt = b.CSER(d, n, bs, R1, R2, H, 0.1, beta, 12, flags=flags)
+    ref = (CSERImpl2Oracle if impl2 else CSEROracle)(d, n, bs, R1, R2, H, 0.1, beta, 12, dtype=np.float32)
+    opt.set_x0(torch.from_numpy(x0).to(DEV)), ref.set_x0(x0)
+    for phase, steps in (("plain", 3), ("replay", 7), ("plain", 3)):
+        if phase == "replay":
+            b.cser_replay_begin(opt.h)
+        for _ in range(steps):
+            g = rng.standard_normal((n, d)).astype(np.float32)
+            gd = torch.from_numpy(g).to(DEV)
+            if phase == "replay":
+                b.cser_step_replayable(opt.h, gd)
+            else:
+                opt.step(gd)
+            ref.step(g)
+            assert opt.t == ref.t
+            assert np.array_equal(opt.state(b.STATE_MASK_G).cpu().numpy(), ref.mask_g), (phase, ref.t)
+        if phase == "replay":
+            assert b.lib().cser_step(opt.h, gd.data_ptr(), None) == -1         # refused in between
+            b.cser_replay_end(opt.h)
+    names = ((b.STATE_X, "x"),) + (() if impl2 else ((b.STATE_E, "e"),)) + (((b.STATE_M, "m"),) if beta else ())
+    for which, name in names:
+        assert np.array_equal(opt.state(which).cpu().numpy(), getattr(ref, name)), name
+    opt.close()
+
+
+def test_step_captured_once_in_a_cuda_graph_and_replayed():
+    w = synth.CONFIGS[2].scaled(d=400_000 + 8, steps=20)
+    R1, R2, H = 4, 2, 3
+    opt = b.CSER(w.d, w.n_workers, w.block_size, R1, R2, H, w.eta, w.beta, 21)
+    ref = CSEROracle(w.d, w.n_workers, w.block_size, R1, R2, H, w.eta, w.beta, 21, dtype=np.float32)
+    x0 = synth.x0(w, DEV)
+    opt.set_x0(x0), ref.set_x0(x0.cpu().numpy())
+    grads = [synth.gradients(w, t, DEV) for t in range(1, w.steps + 1)]
+    static_g = torch.empty_like(grads[0])
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        b.cser_replay_begin(opt.h)
+        static_g.copy_(grads[0])
+        b.cser_step_replayable(opt.h, static_g)                 # iteration 1, eagerly (also warms up)
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side, capture_error_mode="thread_local"):
+        b.cser_step_replayable(opt.h, static_g)                 # captured, not run
+    ref.step(grads[0].cpu().numpy())
+    for t in range(2, w.steps + 1):
+        static_g.copy_(grads[t - 1])
+        graph.replay()
+        ref.step(grads[t - 1].cpu().numpy())
+    torch.cuda.synchronize()
+    assert opt.t == w.steps                                      # read from the device
+    b.cser_replay_end(opt.h)
+    assert opt.t == w.steps
+    for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e"), (b.STATE_M, "m")):
+        assert np.array_equal(opt.state(which).cpu().numpy(), getattr(ref, name)), name
+    opt.step(grads[0])                                           # ordinary steps continue from there
+    ref.step(grads[0].cpu().numpy())
+    assert np.array_equal(opt.state(b.STATE_X).cpu().numpy(), ref.x)
+    opt.close()
+
+
 # ------------------------------------------------------------------ randomized differential test
 def test_random_shapes_parameters_and_flags_against_the_float32_oracle():
     """400 random problems (shape, ratios, reset interval, momentum, flags, injected masks now and
