@@ -150,7 +150,7 @@ def oracle_all_cores(w, seconds=10.0):
     """The same oracle with the columns split over all host cores: one process per core, each
     timing its own slab of whole blocks at the same moment.  Returns (steps/s, description, cores)."""
     import subprocess
-    cores = os.cpu_count() or 1
+    cores = min(os.cpu_count() or 1, 32)       # one Python process per core; keep the memory bounded
     procs = [subprocess.Popen([sys.executable, os.path.abspath(__file__), "--config", str(w_index(w)),
                                "--oracle-slab", str(k), "--oracle-seconds", str(seconds)] +
                               (["--d", str(w.d)] if w.d != base_config(w).d else []),
