@@ -550,6 +550,8 @@ def main():
                        + (" exact-count GRBS" if args.exact_count else ""),
                        "d": w.d, "n_workers": w.n_workers, "block_size": w.block_size,
                        "R1": w.R1, "R2": w.R2, "H": w.H, "eta": w.eta, "beta": w.beta,
+                       "overall_compression_ratio": w.overall_ratio,
+                       "deployment_bytes_per_worker_step": w.comm_bytes_per_worker_step,
                        "parallelism": f"column slabs x{world}, no collective",
                        "l2": f"inputs larger than L2: {alg_bytes / 1e9:.2f} GB touched per step, "
                              f"{r['ring_n']} gradient buffers cycled"},

@@ -36,6 +36,17 @@ class Workload:
     def n_blocks(self):
         return (self.d + self.block_size - 1) // self.block_size
 
+    @property
+    def overall_ratio(self):
+        """Overall compression ratio R_C = 1 / (1/R1 + 1/(R2 H)) (Section 5.1; R1 = 0 means no per-step part)."""
+        inv = (1.0 / self.R1 if self.R1 else 0.0) + 1.0 / (self.R2 * self.H)
+        return 1.0 / inv
+
+    @property
+    def comm_bytes_per_worker_step(self):
+        """fp32 bytes a worker would put on the wire per step in a real deployment (average over H steps)."""
+        return 4.0 * self.d / self.overall_ratio
+
     def scaled(self, d, steps=None):
         """Same hyper-parameters on a shorter vector (for quick tests)."""
         return replace(self, d=int(d), steps=self.steps if steps is None else int(steps),

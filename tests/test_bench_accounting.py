@@ -31,3 +31,15 @@ def test_variants_change_the_count_as_stated():
     assert bench.expected_e_fraction(replace(w, R1=0), False) == 1.0      # C2 = 0: e touched everywhere
     assert bench.expected_e_fraction(replace(w, R1=1, R2=1), True) == 1.0
     assert bench.expected_e_fraction(replace(w, R1=1), False) == 0.0      # everything synchronized: e idle
+
+
+def test_overall_compression_ratio_matches_the_papers_formula_and_table():
+    """Section 5.1: R_C = 1 / (1/R_C2 + 1/(R_C1 H)); Appendix C lists (R_C2, R_C1, H) = (512, 16, 32) for an
+    overall ratio of 256 and (2048, 32, 64) for 1024 (R1 here is the paper's R_C2, R2 its R_C1)."""
+    from dataclasses import replace
+    w = synth.CONFIGS[2]
+    assert abs(replace(w, R1=512, R2=16, H=32).overall_ratio - 256.0) < 1e-9
+    assert abs(replace(w, R1=2048, R2=32, H=64).overall_ratio - 1024.0) < 1e-9
+    assert abs(replace(w, R1=64, R2=8, H=8).overall_ratio - 32.0) < 1e-9
+    assert abs(w.overall_ratio - 1.0 / (1 / 32 + 1 / 256)) < 1e-12
+    assert replace(w, R1=0, R2=4, H=2).overall_ratio == 8.0            # CSER-PL: only the reset is exchanged
