@@ -36,10 +36,13 @@ def test_variants_change_the_count_as_stated():
 def test_overall_compression_ratio_matches_the_papers_formula_and_table():
     """Section 5.1: R_C = 1 / (1/R_C2 + 1/(R_C1 H)); Appendix C lists (R_C2, R_C1, H) = (512, 16, 32) for an
     overall ratio of 256 and (2048, 32, 64) for 1024 (R1 here is the paper's R_C2, R2 its R_C1)."""
+    import os
     from dataclasses import replace
     w = synth.CONFIGS[2]
-    assert abs(replace(w, R1=512, R2=16, H=32).overall_ratio - 256.0) < 1e-9
-    assert abs(replace(w, R1=2048, R2=32, H=64).overall_ratio - 1024.0) < 1e-9
-    assert abs(replace(w, R1=64, R2=8, H=8).overall_ratio - 32.0) < 1e-9
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "table3_cser_hyperparameters.txt")
+    rows = [tuple(int(v) for v in ln.split()) for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 6
+    for overall, R1, R2, H in rows:
+        assert abs(replace(w, R1=R1, R2=R2, H=H).overall_ratio - overall) < 1e-9, (overall, R1, R2, H)
     assert abs(w.overall_ratio - 1.0 / (1 / 32 + 1 / 256)) < 1e-12
     assert replace(w, R1=0, R2=4, H=2).overall_ratio == 8.0            # CSER-PL: only the reset is exchanged
