@@ -498,7 +498,8 @@ def main():
                     "kernel_gbs": ro["roofline"]["achieved"], "kernel_frac_of_measured": ro["roofline"]["frac"]}
 
         def other_workload(c):
-            wo = synth.CONFIGS[c]
+            wo = c if isinstance(c, synth.Workload) else synth.CONFIGS[c]
+            c = 0 if isinstance(c, synth.Workload) else c
             free, _ = torch.cuda.mem_get_info()
             if free < wo.n_workers * wo.d * 4 * 6.5:
                 return "skipped: not enough free device memory"
@@ -521,6 +522,8 @@ def main():
         guarded(w.name + " implementation II (no error array, 20 B per element-worker)", lambda: variant("impl2"))
         for c in (1, 3, 4, 5):
             guarded(synth.CONFIGS[c].name, lambda c=c: other_workload(c))
+        for rc, wt in synth.PAPER_TUNED.items():     # the paper's tuned (R_C2, R_C1, H) per overall ratio
+            guarded(wt.name, lambda wt=wt: other_workload(wt))
 
         def l2_resident():
             global L2_RESIDENT

@@ -67,6 +67,13 @@ CONFIGS = {
                 "iid", 0.0, 1e-3 ** 0.5),
 }
 
+# The paper's own tuned settings for WRN-40-8 (Appendix C, CSER rows), on the WRN-40-8-sized vector:
+# overall ratio -> (R1 = its R_C2, R2 = its R_C1, H).
+PAPER_TUNED = {
+    rc: replace(CONFIGS[2], name=f"wrn40x8_paper_tuned_RC{rc}_R{r1}_{r2}_H{h}", R1=r1, R2=r2, H=h)
+    for rc, (r1, r2, h) in {32: (64, 8, 8), 256: (512, 16, 32), 1024: (2048, 32, 64)}.items()
+}
+
 
 def _gen(device, *words):
     g = torch.Generator(device=device)
