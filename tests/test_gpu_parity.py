@@ -487,6 +487,31 @@ def test_learning_rate_schedule_and_column_reads():
     opt.close()
 
 
+def test_two_handles_stepping_concurrently_on_two_streams():
+    w = synth.CONFIGS[2].scaled(d=1_000_000, steps=12)
+    seeds = (31, 32)
+    ref = [b.CSER(w.d, w.n_workers, w.block_size, 8, 4, 3, w.eta, w.beta, s) for s in seeds]
+    par = [b.CSER(w.d, w.n_workers, w.block_size, 8, 4, 3, w.eta, w.beta, s) for s in seeds]
+    x0 = synth.x0(w, DEV)
+    for h in ref + par:
+        h.set_x0(x0)
+    grads = [synth.gradients(w, t, DEV) for t in range(1, w.steps + 1)]
+    torch.cuda.synchronize()
+    for g in grads:                                   # one after the other
+        for h in ref:
+            h.step(g)
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for g in grads:                                   # interleaved on two streams, no synchronization between
+        for h, st in zip(par, streams):
+            with torch.cuda.stream(st):
+                h.step(g)
+    torch.cuda.synchronize()
+    for a, c in zip(ref, par):
+        for which in (b.STATE_X, b.STATE_E, b.STATE_M):
+            assert torch.equal(a.state(which), c.state(which))
+    [h.close() for h in ref + par]
+
+
 def test_l2_resident_state_gives_the_same_results():
     w = synth.CONFIGS[1].scaled(d=300_000, steps=9)          # 9.6 MB of state: fits the L2 set-aside
     a = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, 3)
