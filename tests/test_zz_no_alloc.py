@@ -52,3 +52,32 @@ def test_noalloc_rejects_vectors_beyond_its_built_in_scratch():
     assert rc == -1 and "exceed" in b.cser_last_error()
     rc = L.cser_step_noalloc(8, 1, 4, 2, 2, 2, 0.1, 0.0, 0, 0, z.data_ptr(), z.data_ptr(), z.data_ptr(), None, None)
     assert rc == -1                                 # t is 1-based
+
+
+@pytest.mark.parametrize("d,n,bs,beta", [(10_000 + 36, 8, 256, 0.9), (1001, 3, 7, 0.9), (4099, 5, 64, 0.0),
+                                         (70_000, 16, 1024, 0.9)])
+def test_kernels_never_write_outside_the_arrays_they_are_given(d, n, bs, beta):
+    """Guard bands: with the caller-owned arrays of the allocation-free entry point, x, e, m and the
+    gradients sit inside larger buffers filled with a sentinel; after steps through every kernel path
+    (plain and reset steps, selected and unselected blocks, ragged last block) the sentinels around
+    each array must be untouched."""
+    torch.cuda.set_device(0)
+    pad, sentinel = 4096, 12345.0
+    total = n * d
+
+    def guarded():
+        buf = torch.full((total + 2 * pad,), sentinel, dtype=torch.float32, device=DEV)
+        return buf, buf[pad:pad + total].view(n, d)
+
+    (bx, x), (be, e), (bm, m), (bg, g) = guarded(), guarded(), guarded(), guarded()
+    x.copy_(torch.randn(d, device=DEV)[None, :].expand(n, d))
+    e.zero_(), m.zero_()
+    for t in range(1, 9):                                   # H = 2: four reset steps
+        g.copy_(torch.randn((n, d), device=DEV))
+        b.cser_step_noalloc(d, n, bs, 2, 2, 2, 0.1, beta, 5, t, g, x, e, m if beta else None)
+    torch.cuda.synchronize()
+    for name, buf in (("x", bx), ("e", be), ("m", bm), ("g", bg)):
+        assert bool((buf[:pad] == sentinel).all()) and bool((buf[pad + total:] == sentinel).all()), name
+    assert bool(torch.isfinite(x).all()) and bool((x != sentinel).any())
+    if not beta:
+        assert bool((m == 0).all())                         # no momentum: m is never touched
