@@ -750,6 +750,15 @@ def test_errors_are_reported_not_raised_on_the_device():
     assert L.cser_read_state(opt.h, b.STATE_X, ctypes.c_void_p(small.data_ptr()), 40, None) == -4
     assert L.cser_read_state(opt.h, b.STATE_M, ctypes.c_void_p(small.data_ptr()), 40, None) == -1
     assert L.cser_read_state(opt.h, 17, ctypes.c_void_p(small.data_ptr()), 40, None) == -1
+    dev_g = torch.zeros((2, 100 + 1), device=DEV)
+    assert L.cser_step(opt.h, ctypes.c_void_p(dev_g.data_ptr() + 2), None) == -1    # not 4-byte aligned
+    assert "aligned" in b.cser_last_error()
+    assert L.cser_write_state(opt.h, b.STATE_X, ctypes.c_void_p(small.data_ptr()), 40, None) == -4
+    assert L.cser_write_state(opt.h, b.STATE_MASK_G, ctypes.c_void_p(small.data_ptr()), 10, None) == -1
+    assert L.cser_debug_set_masks(opt.h, None, None, None) == -1
+    assert L.cser_set_x0(opt.h, None, None) == -1
+    assert L.cser_grbs_mask(0, 1, 2, 0, 10, 4, ctypes.c_void_p(small.data_ptr()), None) == -1   # bad compressor id
+    assert L.cser_last_kernel_ms(opt.h, None, None) == -1                                # nothing timed yet
     assert opt.t == 0                                 # failed calls did not advance the step counter
     opt.step(torch.zeros((2, 100), device=DEV))
     assert opt.t == 1
