@@ -85,7 +85,7 @@ struct cser_ctx {
     const uint32_t *pre_count = nullptr;
     bool walk_all = false;                           // masks were injected: no estimate of the selected count
     // replayable steps (cser_replay_begin .. cser_replay_end): the iteration lives on the device
-    StepCtl *ctl = nullptr;
+    ReplayCtl *ctl = nullptr;
     bool replay = false;
     // worker-sharded mode (cser_create_wshard): n = local workers, n_total = all ranks' workers
     int n_total = 0;
@@ -204,7 +204,9 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     if (grid_ll > 0x7fffffffll) return fail(CSER_ERR_INVALID, "n_workers * d too large for one launch");
     StepParams Q = P;
     Q.tiles = (unsigned)tiles;
-    Q.ctl = h->replay ? h->ctl : nullptr;
+    Q.rctl = h->replay ? h->ctl : nullptr;
+    Q.sel_stride = h->replay ? h->B : 0;
+    if (h->replay) Q.mask_g = h->sb[0].mask_g, Q.mask_r = h->sb[0].mask_r, Q.list = h->sb[0].list;
     if (h->replay) is_reset = true;   // the reset variants decide on the device whether this step resets
     const unsigned grid = (unsigned)grid_ll;
     // Grid of the selected-block kernel: the count lives on the device, so size the grid for
@@ -285,6 +287,16 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     h->launches += stream_any ? 2 : 1;
     CU_TRY(lerr);
     CU_TRY(cudaGetLastError());
+    if (h->replay) {
+        // the following iteration's masks and list, behind the selected-block kernel
+        const unsigned sgrid = (unsigned)((h->B + 255) / 256);
+        grbs_select_replay_kernel<<<sgrid, 256, 0, ws>>>(h->ctl, h->sb[0].mask_g, h->sb[0].mask_r, h->sb[0].list,
+                                                         h->B, h->B, h->block_begin,
+                                                         (uint32_t)(h->seed & 0xffffffffu), (uint32_t)(h->seed >> 32),
+                                                         h->R1, h->R2, (uint32_t)h->H);
+        h->launches++;
+        CU_TRY(cudaGetLastError());
+    }
     if (fork) {
         int rc = CSER_OK;
         if (prefetch) {
@@ -309,7 +321,7 @@ int launch_step(cser_ctx *h, const float *grad, long long col0, long long col1, 
     P.g = grad, P.x = h->x, P.e = h->e, P.m = h->m;
     P.mask_g = h->mask_g, P.mask_r = h->mask_r;
     P.list = h->sel_list, P.count = h->cur_count;
-    P.tiles = 0, P.ctl = nullptr;
+    P.tiles = 0, P.rctl = nullptr, P.sel_stride = 0;
     P.d = h->d, P.n = h->n;
     P.eta = h->eta, P.beta = h->beta, P.n_f = (float)h->n;
     const bool v4 = h->vec4 && ((uintptr_t)grad % 16 == 0) && (col0 % 4 == 0) &&
@@ -407,12 +419,15 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
         if (with_e_) h->e = reinterpret_cast<float *>(p), p += arr_bytes;
         if (beta != 0.f) h->m = reinterpret_cast<float *>(p);
     }
-    for (auto &sb : h->sb) {
-        if (er == cudaSuccess) er = cudaMalloc(&sb.mask_g, (size_t)B);
-        if (er == cudaSuccess) er = cudaMalloc(&sb.mask_r, (size_t)B);
-        if (er == cudaSuccess) er = cudaMalloc(&sb.list, (size_t)B * sizeof(uint32_t));
-        if (er == cudaSuccess) er = cudaMemset(sb.mask_g, 0, (size_t)B);
-        if (er == cudaSuccess) er = cudaMemset(sb.mask_r, 0, (size_t)B);
+    // the two buffer sets lie B entries apart in one allocation per kind
+    if (er == cudaSuccess) er = cudaMalloc(&h->sb[0].mask_g, 2 * (size_t)B);
+    if (er == cudaSuccess) er = cudaMalloc(&h->sb[0].mask_r, 2 * (size_t)B);
+    if (er == cudaSuccess) er = cudaMalloc(&h->sb[0].list, 2 * (size_t)B * sizeof(uint32_t));
+    if (er == cudaSuccess) er = cudaMemset(h->sb[0].mask_g, 0, 2 * (size_t)B);
+    if (er == cudaSuccess) er = cudaMemset(h->sb[0].mask_r, 0, 2 * (size_t)B);
+    if (er == cudaSuccess) {
+        h->sb[1].mask_g = h->sb[0].mask_g + B, h->sb[1].mask_r = h->sb[0].mask_r + B;
+        h->sb[1].list = h->sb[0].list + B;
     }
     if (er == cudaSuccess) er = cudaMemset(h->state_base, 0, h->state_bytes);
     if (er == cudaSuccess && (flags & CSER_FLAG_L2_RESIDENT)) {
@@ -434,8 +449,8 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
     if (er == cudaSuccess && h->exact) er = cudaMalloc(&h->exact_scratch, sizeof(ExactScratch));
     if (er == cudaSuccess && h->exact) er = cudaMemset(h->exact_scratch, 0, sizeof(ExactScratch));
     if (er == cudaSuccess && h->exact) er = cudaMalloc(&h->exact_words, 2 * (size_t)B * sizeof(uint32_t));
-    if (er == cudaSuccess) er = cudaMalloc(&h->ctl, sizeof(StepCtl));
-    if (er == cudaSuccess) er = cudaMemset(h->ctl, 0, sizeof(StepCtl));
+    if (er == cudaSuccess) er = cudaMalloc(&h->ctl, sizeof(ReplayCtl));
+    if (er == cudaSuccess) er = cudaMemset(h->ctl, 0, sizeof(ReplayCtl));
     if (er == cudaSuccess) er = cudaMalloc(&h->sel_count, 3 * sizeof(uint32_t));
     if (er == cudaSuccess) er = cudaMemset(h->sel_count, 0, 3 * sizeof(uint32_t));
     if (er == cudaSuccess) activate_selection(h, 0, h->sel_count, true);
@@ -477,7 +492,7 @@ void cser_destroy(cser_handle h) {
         cudaGetLastError();
     }
     cudaFree(h->state_base);
-    for (auto &sb : h->sb) cudaFree(sb.mask_g), cudaFree(sb.mask_r), cudaFree(sb.list);
+    cudaFree(h->sb[0].mask_g), cudaFree(h->sb[0].mask_r), cudaFree(h->sb[0].list);
     cudaFree(h->x0_stage), cudaFree(h->g_stage);
     cudaFree(h->sel_count), cudaFree(h->exact_scratch), cudaFree(h->exact_words), cudaFree(h->ctl);
     cudaFree(h->pos_g), cudaFree(h->pos_r), cudaFree(h->olist_g), cudaFree(h->olist_r);
@@ -601,10 +616,19 @@ int cser_read_state(cser_handle h, int which, void *dst, size_t dst_bytes, void 
     if (int rc = state_piece(h, which, &src, &bytes)) return rc;
     if (dst_bytes < bytes)
         return fail(CSER_ERR_TOO_SMALL, "cser_read_state: need %zu bytes, got %zu", bytes, dst_bytes);
+    if (h->replay && (which == CSER_STATE_MASK_G || which == CSER_STATE_MASK_R)) {
+        // which buffer set is current is known on the device only
+        CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+        ReplayCtl c = {};
+        CU_TRY(cudaMemcpy(&c, h->ctl, sizeof(c), cudaMemcpyDeviceToHost));
+        src = which == CSER_STATE_MASK_G ? h->sb[c.cur].mask_g : h->sb[c.cur].mask_r;
+    }
     if (which == CSER_STATE_T) {
         if (h->replay) {   // the counter lives on the device while steps are replayable
             CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));
-            CU_TRY(cudaMemcpy(dst, &h->ctl->t, sizeof(uint64_t), cudaMemcpyDefault));
+            ReplayCtl c = {};
+            CU_TRY(cudaMemcpy(&c, h->ctl, sizeof(c), cudaMemcpyDeviceToHost));
+            CU_TRY(cudaMemcpy(dst, &c.c[c.cur].t, sizeof(uint64_t), cudaMemcpyDefault));
             return CSER_OK;
         }
         CU_TRY(cudaMemcpy(dst, &h->t, sizeof(uint64_t), cudaMemcpyDefault));
@@ -811,12 +835,20 @@ int cser_replay_begin(cser_handle h, void *stream) {
     if (h->exact || h->n_total > 0 || h->masks_injected)
         return fail(CSER_ERR_INVALID,
                     "cser_replay_begin: not available with exact-count masks, worker sharding or injected masks");
-    StepCtl c = {};
-    c.t = h->t;
-    CU_TRY(cudaMemcpyAsync(h->ctl, &c, sizeof(c), cudaMemcpyHostToDevice, (cudaStream_t)stream));
-    CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));   // c is on this function's stack
+    cudaStream_t s = (cudaStream_t)stream;
+    ReplayCtl c = {};
+    c.c[0].t = h->t;           // block 0 stands for the iteration already done; cur = 0
+    CU_TRY(cudaMemcpyAsync(h->ctl, &c, sizeof(c), cudaMemcpyHostToDevice, s));
+    CU_TRY(cudaStreamSynchronize(s));   // c is on this function's stack
+    // masks and list of iteration t + 1 into buffer set 1, published in block 1
+    const unsigned grid = (unsigned)((h->B + 255) / 256);
+    grbs_select_replay_kernel<<<grid, 256, 0, s>>>(h->ctl, h->sb[0].mask_g, h->sb[0].mask_r, h->sb[0].list, h->B,
+                                                   h->B, h->block_begin, (uint32_t)(h->seed & 0xffffffffu),
+                                                   (uint32_t)(h->seed >> 32), h->R1, h->R2, (uint32_t)h->H);
+    h->launches++;
+    CU_TRY(cudaGetLastError());
     h->pre_valid = false;
-    activate_selection(h, 0, nullptr, true);
+    h->walk_all = false;
     h->replay = true;
     return CSER_OK;
 }
@@ -830,13 +862,9 @@ int cser_step_replayable(cser_handle h, const float *grad, void *stream) {
     }
     if ((uintptr_t)grad % 4 != 0) return fail(CSER_ERR_INVALID, "cser_step_replayable: grad is not 4-byte aligned");
     cudaStream_t s = (cudaStream_t)stream;
-    const unsigned grid = (unsigned)((h->B + 255) / 256);
-    grbs_select_replay_kernel<<<grid, 256, 0, s>>>(h->ctl, h->sb[0].mask_g, h->sb[0].mask_r, h->sb[0].list, h->B,
-                                                   h->block_begin, (uint32_t)(h->seed & 0xffffffffu),
-                                                   (uint32_t)(h->seed >> 32), h->R1, h->R2, (uint32_t)h->H);
+    replay_advance_kernel<<<1, 1, 0, s>>>(h->ctl);       // the iteration prepared last step becomes current
     h->launches++;
     CU_TRY(cudaGetLastError());
-    h->walk_all = false;
     return launch_step(h, grad, 0, h->d, true, s, true);
 }
 
@@ -844,12 +872,12 @@ int cser_replay_end(cser_handle h, void *stream) {
     if (int rc = check_handle(h)) return rc;
     if (!h->replay) return fail(CSER_ERR_INVALID, "cser_replay_end: not begun");
     CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));
-    StepCtl c = {};
+    ReplayCtl c = {};
     CU_TRY(cudaMemcpy(&c, h->ctl, sizeof(c), cudaMemcpyDeviceToHost));
-    h->t = c.t;
+    h->t = c.c[c.cur].t;
     h->replay = false;
     h->pre_valid = false;
-    if (c.reset) h->last_mask_r = h->sb[0].mask_r;
+    activate_selection(h, (int)c.cur, h->sel_count, c.c[c.cur].reset != 0);   // masks of the last iteration
     return CSER_OK;
 }
 

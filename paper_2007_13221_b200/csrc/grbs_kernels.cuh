@@ -181,28 +181,44 @@ grbs_select_kernel(uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r,
 
 // ------------------------------------------------------------------ replayable steps
 // For a step that is captured once in a CUDA graph and replayed, the iteration number cannot
-// be a launch argument.  It lives in this device-side block instead: the select kernel of a
-// step works on iteration ctl->t + 1 and its last CTA to finish publishes it (t, whether it
-// resets), after which the step kernels of the same step read it.  The two list counters are
-// used alternately by the parity of t.
+// be a launch argument.  It lives in device memory instead, in two blocks used alternately:
+// c[cur] describes the iteration the step kernels are working on; while they run, the select
+// kernel prepares iteration c[cur].t + 1 in the other buffer set and publishes it in
+// c[cur ^ 1] (its last CTA to finish does so: a counter, no waiting).  A one-thread kernel at
+// the start of every step flips cur.  Nothing ever waits on anything.
 struct StepCtl {
-    unsigned long long t;      // last iteration whose select kernel has completed
-    uint32_t reset;            // that iteration is a reset step
-    uint32_t done;             // CTAs of the running select kernel that have finished
-    uint32_t count[2];         // selected-block counters, indexed by t & 1
+    unsigned long long t;      // the iteration this block describes
+    uint32_t reset;            // it is a reset step
+    uint32_t done;             // CTAs of the select kernel filling this block that have finished
+    uint32_t count;            // blocks in this iteration's list
+    uint32_t pad;
+};
+struct ReplayCtl {
+    StepCtl c[2];
+    uint32_t cur;
 };
 
+__global__ void replay_advance_kernel(ReplayCtl *R) {
+    const uint32_t old = R->cur;
+    R->c[old].count = 0;       // the step that used this block has finished; it is filled next
+    R->c[old].done = 0;
+    R->cur = old ^ 1u;
+}
+
+// mask_g / mask_r / list point at buffer set 0; set 1 lies sel_stride entries further.
 __global__ void __launch_bounds__(256)
-grbs_select_replay_kernel(StepCtl *ctl, uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r,
-                          uint32_t *__restrict__ list, long long B, long long block_begin, uint32_t k0,
-                          uint32_t k1, uint32_t R_g, uint32_t R_r, uint32_t H) {
-    // Every thread reads t before any CTA can publish the new one: publishing needs all CTAs done.
-    const unsigned long long t = *(volatile unsigned long long *)&ctl->t + 1ull;
+grbs_select_replay_kernel(ReplayCtl *R, uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r,
+                          uint32_t *__restrict__ list, long long sel_stride, long long B,
+                          long long block_begin, uint32_t k0, uint32_t k1, uint32_t R_g, uint32_t R_r,
+                          uint32_t H) {
+    const uint32_t cur = R->cur, target = cur ^ 1u;
+    const unsigned long long t = R->c[cur].t + 1ull;
     const bool is_reset = (t % H) == 0;
     const uint32_t t_lo = (uint32_t)(t & 0xffffffffu), t_hi = (uint32_t)(t >> 32);
-    uint32_t *count = &ctl->count[t & 1];
+    StepCtl *out = &R->c[target];
+    mask_g += (size_t)target * sel_stride, mask_r += (size_t)target * sel_stride;
+    list += (size_t)target * sel_stride;
     const long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (b == 0) ctl->count[(t + 1) & 1] = 0;     // the previous step's kernels have finished with it
     bool sg = false, sr = false;
     if (b < B) {
         const uint32_t gb = (uint32_t)(block_begin + b);
@@ -220,18 +236,16 @@ grbs_select_replay_kernel(StepCtl *ctl, uint8_t *__restrict__ mask_g, uint8_t *_
         const unsigned lane = threadIdx.x & 31;
         const int leader = __ffs(ballot) - 1;
         unsigned base = 0;
-        if ((int)lane == leader) base = atomicAdd(count, (unsigned)__popc(ballot));
+        if ((int)lane == leader) base = atomicAdd(&out->count, (unsigned)__popc(ballot));
         base = __shfl_sync(0xffffffffu, base, leader);
         if (need) list[base + __popc(ballot & ((1u << lane) - 1u))] = (uint32_t)b;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
-        if (atomicAdd(&ctl->done, 1u) == gridDim.x - 1) {   // last CTA: everything above is visible
-            ctl->reset = is_reset ? 1u : 0u;
-            ctl->done = 0;
-            __threadfence();
-            *(volatile unsigned long long *)&ctl->t = t;
+        if (atomicAdd(&out->done, 1u) == gridDim.x - 1) {   // last CTA: publish the iteration
+            out->t = t;
+            out->reset = is_reset ? 1u : 0u;
         }
     }
 }

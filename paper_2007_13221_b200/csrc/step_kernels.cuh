@@ -47,7 +47,8 @@ struct StepParams {
     const uint8_t *mask_g, *mask_r;
     const uint32_t *list;    // blocks selected by either mask this step
     const uint32_t *count;   // how many
-    const StepCtl *ctl;      // replayable steps: iteration, reset flag and counters on the device (else NULL)
+    const ReplayCtl *rctl;   // replayable steps: iteration, reset flag, list length and buffer set on the device
+    long long sel_stride;    // ... where buffer set 1 lies that many entries after set 0 (else NULL, 0)
     long long d;             // elements per row
     long long cols_total;    // vector columns per row
     long long c_begin;       // first vector column handled by this launch
@@ -109,8 +110,12 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
     constexpr int UA = CSER_WALK_UA(MOM);                      // pass A: g (+ m)
     constexpr int UB = CSER_WALK_UB(RESET && ERR);             // pass B: x (+ e on reset steps)
     constexpr int UF = CSER_WALK_UF;                           // last pass: x only
-    const uint32_t n_listed = DENSE ? 0u : (P.ctl ? P.ctl->count[P.ctl->t & 1] : *P.count);
-    const bool reset_on = RESET && (P.ctl ? P.ctl->reset != 0 : true);
+    const uint32_t rcur = P.rctl ? P.rctl->cur : 0u;
+    const uint8_t *__restrict__ mask_g = P.mask_g + (size_t)rcur * P.sel_stride;
+    const uint8_t *__restrict__ mask_r = P.mask_r + (size_t)rcur * P.sel_stride;
+    const uint32_t *__restrict__ list = P.list + (size_t)rcur * P.sel_stride;
+    const uint32_t n_listed = DENSE ? 0u : (P.rctl ? P.rctl->c[rcur].count : *P.count);
+    const bool reset_on = RESET && (P.rctl ? P.rctl->c[rcur].reset != 0 : true);
     const unsigned long long total =
         DENSE ? (unsigned long long)(P.c_end - P.c_begin) : (unsigned long long)n_listed * P.bsv;
     const long long d = P.d;
@@ -126,12 +131,12 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
         } else {
             const unsigned long long entry =
                 (total <= 0xffffffffull) ? (unsigned long long)((uint32_t)f / P.bsv) : f / P.bsv;
-            blk = P.list[entry];
+            blk = list[entry];
             c = (long long)blk * P.bsv + (long long)(f - entry * P.bsv);
             if (c >= P.cols_total || c < P.c_begin || c >= P.c_end) continue;
         }
-        const bool sg = P.mask_g[blk] != 0;
-        const bool sr = reset_on ? (P.mask_r[blk] != 0) : false;
+        const bool sg = mask_g[blk] != 0;
+        const bool sr = reset_on ? (mask_r[blk] != 0) : false;
         if constexpr (DENSE) {
             if (!sg && !sr) continue;
         }
@@ -305,8 +310,11 @@ __global__ void __launch_bounds__(kStepThreads, 8) cser_stream_kernel(const Step
     if (c >= P.c_end) return;
     const long long b = (P.c_end <= 0xffffffffll) ? (long long)((uint32_t)c / P.bsv)
                                                   : (long long)((unsigned long long)c / P.bsv);
-    if (P.mask_g[b] != 0) return;
-    if (RESET && P.mask_r[b] != 0 && (P.ctl == nullptr || P.ctl->reset != 0)) return;
+    const uint32_t rcur = P.rctl ? P.rctl->cur : 0u;
+    if (P.mask_g[(size_t)rcur * P.sel_stride + b] != 0) return;
+    if (RESET && P.mask_r[(size_t)rcur * P.sel_stride + b] != 0 &&
+        (P.rctl == nullptr || P.rctl->c[rcur].reset != 0))
+        return;
     // C(p) = 0, so p' = r = p (Algorithm 3 lines 4-8): x_i -= p_i, e_i -= p_i (no e array in
     // implementation II).
     const long long o = (long long)row * P.d + c * V;
