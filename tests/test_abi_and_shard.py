@@ -33,6 +33,26 @@ def test_library_builds_loads_and_exports_every_declared_symbol():
     assert L.cser_last_error() == b""
 
 
+def test_header_is_plain_c_and_the_library_links_from_c(tmp_path):
+    import subprocess
+    import __graft_entry__
+    __graft_entry__.build()
+    pkg = os.path.join(ROOT, "paper_2007_13221_b200")
+    exe = str(tmp_path / "abi_c_check")
+    cmd = ["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+           os.path.join(ROOT, "tests", "abi_c_check.c"), "-o", exe, "-L", pkg, "-l:libcser.so",
+           "-Wl,-rpath," + pkg]
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    assert res.returncode == 0, res.stderr
+    run = subprocess.run([exe], capture_output=True, text=True)
+    assert run.returncode == 0, (run.returncode, run.stdout, run.stderr)
+    # every function the header declares is exercised by the C program
+    header = re.sub(r"/\*.*?\*/", "", open(os.path.join(ROOT, "include", "cser.h")).read(), flags=re.S)
+    declared = set(re.findall(r"\b(cser_[a-z0-9_]+)\s*\(", header))
+    used = set(re.findall(r"\b(cser_[a-z0-9_]+)\b", open(os.path.join(ROOT, "tests", "abi_c_check.c")).read()))
+    assert declared <= used, declared - used
+
+
 def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
     from paper_2007_13221_b200 import binding
     monkeypatch.setattr(binding, "_lib", None)
