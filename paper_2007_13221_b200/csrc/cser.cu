@@ -205,7 +205,6 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     StepParams Q = P;
     Q.tiles = (unsigned)tiles;
     Q.rctl = h->replay ? h->ctl : nullptr;
-    Q.sel_stride = h->replay ? h->B : 0;
     if (h->replay) Q.mask_g = h->sb[0].mask_g, Q.mask_r = h->sb[0].mask_r, Q.list = h->sb[0].list;
     if (h->replay) is_reset = true;   // the reset variants decide on the device whether this step resets
     const unsigned grid = (unsigned)grid_ll;
@@ -321,7 +320,7 @@ int launch_step(cser_ctx *h, const float *grad, long long col0, long long col1, 
     P.g = grad, P.x = h->x, P.e = h->e, P.m = h->m;
     P.mask_g = h->mask_g, P.mask_r = h->mask_r;
     P.list = h->sel_list, P.count = h->cur_count;
-    P.tiles = 0, P.rctl = nullptr, P.sel_stride = 0;
+    P.tiles = 0, P.rctl = nullptr;
     P.d = h->d, P.n = h->n;
     P.eta = h->eta, P.beta = h->beta, P.n_f = (float)h->n;
     const bool v4 = h->vec4 && ((uintptr_t)grad % 16 == 0) && (col0 % 4 == 0) &&
@@ -616,19 +615,14 @@ int cser_read_state(cser_handle h, int which, void *dst, size_t dst_bytes, void 
     if (int rc = state_piece(h, which, &src, &bytes)) return rc;
     if (dst_bytes < bytes)
         return fail(CSER_ERR_TOO_SMALL, "cser_read_state: need %zu bytes, got %zu", bytes, dst_bytes);
-    if (h->replay && (which == CSER_STATE_MASK_G || which == CSER_STATE_MASK_R)) {
-        // which buffer set is current is known on the device only
-        CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));
-        ReplayCtl c = {};
-        CU_TRY(cudaMemcpy(&c, h->ctl, sizeof(c), cudaMemcpyDeviceToHost));
-        src = which == CSER_STATE_MASK_G ? h->sb[c.cur].mask_g : h->sb[c.cur].mask_r;
-    }
+    if (h->replay && (which == CSER_STATE_MASK_G || which == CSER_STATE_MASK_R))
+        src = which == CSER_STATE_MASK_G ? h->sb[0].mask_g : h->sb[0].mask_r;   // set 0 is the current one
     if (which == CSER_STATE_T) {
         if (h->replay) {   // the counter lives on the device while steps are replayable
             CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));
             ReplayCtl c = {};
             CU_TRY(cudaMemcpy(&c, h->ctl, sizeof(c), cudaMemcpyDeviceToHost));
-            CU_TRY(cudaMemcpy(dst, &c.c[c.cur].t, sizeof(uint64_t), cudaMemcpyDefault));
+            CU_TRY(cudaMemcpy(dst, &c.c[0].t, sizeof(uint64_t), cudaMemcpyDefault));
             return CSER_OK;
         }
         CU_TRY(cudaMemcpy(dst, &h->t, sizeof(uint64_t), cudaMemcpyDefault));
@@ -837,7 +831,7 @@ int cser_replay_begin(cser_handle h, void *stream) {
                     "cser_replay_begin: not available with exact-count masks, worker sharding or injected masks");
     cudaStream_t s = (cudaStream_t)stream;
     ReplayCtl c = {};
-    c.c[0].t = h->t;           // block 0 stands for the iteration already done; cur = 0
+    c.c[0].t = h->t;           // block 0 stands for the iteration already done
     CU_TRY(cudaMemcpyAsync(h->ctl, &c, sizeof(c), cudaMemcpyHostToDevice, s));
     CU_TRY(cudaStreamSynchronize(s));   // c is on this function's stack
     // masks and list of iteration t + 1 into buffer set 1, published in block 1
@@ -862,7 +856,9 @@ int cser_step_replayable(cser_handle h, const float *grad, void *stream) {
     }
     if ((uintptr_t)grad % 4 != 0) return fail(CSER_ERR_INVALID, "cser_step_replayable: grad is not 4-byte aligned");
     cudaStream_t s = (cudaStream_t)stream;
-    replay_advance_kernel<<<1, 1, 0, s>>>(h->ctl);       // the iteration prepared last step becomes current
+    // the iteration prepared during the last step becomes the current one
+    replay_advance_kernel<<<(unsigned)((h->B + 255) / 256), 256, 0, s>>>(h->ctl, h->sb[0].mask_g, h->sb[0].mask_r,
+                                                                         h->sb[0].list, h->B, h->B);
     h->launches++;
     CU_TRY(cudaGetLastError());
     return launch_step(h, grad, 0, h->d, true, s, true);
@@ -874,10 +870,10 @@ int cser_replay_end(cser_handle h, void *stream) {
     CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));
     ReplayCtl c = {};
     CU_TRY(cudaMemcpy(&c, h->ctl, sizeof(c), cudaMemcpyDeviceToHost));
-    h->t = c.c[c.cur].t;
+    h->t = c.c[0].t;
     h->replay = false;
     h->pre_valid = false;
-    activate_selection(h, (int)c.cur, h->sel_count, c.c[c.cur].reset != 0);   // masks of the last iteration
+    activate_selection(h, 0, h->sel_count, c.c[0].reset != 0);   // set 0 holds the masks of the last iteration
     return CSER_OK;
 }
 

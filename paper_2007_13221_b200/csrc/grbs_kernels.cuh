@@ -181,11 +181,12 @@ grbs_select_kernel(uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r,
 
 // ------------------------------------------------------------------ replayable steps
 // For a step that is captured once in a CUDA graph and replayed, the iteration number cannot
-// be a launch argument.  It lives in device memory instead, in two blocks used alternately:
-// c[cur] describes the iteration the step kernels are working on; while they run, the select
-// kernel prepares iteration c[cur].t + 1 in the other buffer set and publishes it in
-// c[cur ^ 1] (its last CTA to finish does so: a counter, no waiting).  A one-thread kernel at
-// the start of every step flips cur.  Nothing ever waits on anything.
+// be a launch argument.  It lives in device memory instead.  Block c[0] and buffer set 0
+// describe the iteration the step kernels are working on; while they run, the select kernel
+// prepares iteration c[0].t + 1 in buffer set 1 and publishes it in c[1] (its last CTA to
+// finish does so: a counter, no waiting).  A small kernel at the start of every step copies
+// set 1 and c[1] over set 0 and c[0].  Nothing ever waits on anything, and the step kernels
+// read their masks from the same place as in an ordinary step.
 struct StepCtl {
     unsigned long long t;      // the iteration this block describes
     uint32_t reset;            // it is a reset step
@@ -194,30 +195,45 @@ struct StepCtl {
     uint32_t pad;
 };
 struct ReplayCtl {
-    StepCtl c[2];
-    uint32_t cur;
+    StepCtl c[2];              // [0] current, [1] prepared for the next step
 };
 
-__global__ void replay_advance_kernel(ReplayCtl *R) {
-    const uint32_t old = R->cur;
-    R->c[old].count = 0;       // the step that used this block has finished; it is filled next
-    R->c[old].done = 0;
-    R->cur = old ^ 1u;
+// Buffer set 1 lies `stride` entries after set 0.  One thread per block.
+__global__ void __launch_bounds__(256)
+replay_advance_kernel(ReplayCtl *R, uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r,
+                      uint32_t *__restrict__ list, long long stride, long long B) {
+    const long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t count = R->c[1].count, reset = R->c[1].reset;
+    const unsigned long long t = R->c[1].t;
+    if (b < B) {
+        mask_g[b] = mask_g[stride + b];
+        if (reset) mask_r[b] = mask_r[stride + b];
+        if (b < count) list[b] = list[stride + b];
+    }
+    // the last CTA to finish moves the control block over and re-arms the other one
+    __shared__ bool last;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        last = atomicAdd(&R->c[0].done, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (last && threadIdx.x == 0) {
+        R->c[0].t = t, R->c[0].reset = reset, R->c[0].count = count, R->c[0].done = 0;
+        R->c[1].count = 0, R->c[1].done = 0;
+    }
 }
 
-// mask_g / mask_r / list point at buffer set 0; set 1 lies sel_stride entries further.
 __global__ void __launch_bounds__(256)
 grbs_select_replay_kernel(ReplayCtl *R, uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r,
-                          uint32_t *__restrict__ list, long long sel_stride, long long B,
+                          uint32_t *__restrict__ list, long long stride, long long B,
                           long long block_begin, uint32_t k0, uint32_t k1, uint32_t R_g, uint32_t R_r,
                           uint32_t H) {
-    const uint32_t cur = R->cur, target = cur ^ 1u;
-    const unsigned long long t = R->c[cur].t + 1ull;
+    const unsigned long long t = R->c[0].t + 1ull;      // c[0] does not change while this kernel runs
     const bool is_reset = (t % H) == 0;
     const uint32_t t_lo = (uint32_t)(t & 0xffffffffu), t_hi = (uint32_t)(t >> 32);
-    StepCtl *out = &R->c[target];
-    mask_g += (size_t)target * sel_stride, mask_r += (size_t)target * sel_stride;
-    list += (size_t)target * sel_stride;
+    StepCtl *out = &R->c[1];
+    mask_g += stride, mask_r += stride, list += stride;
     const long long b = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     bool sg = false, sr = false;
     if (b < B) {

@@ -47,8 +47,7 @@ struct StepParams {
     const uint8_t *mask_g, *mask_r;
     const uint32_t *list;    // blocks selected by either mask this step
     const uint32_t *count;   // how many
-    const ReplayCtl *rctl;   // replayable steps: iteration, reset flag, list length and buffer set on the device
-    long long sel_stride;    // ... where buffer set 1 lies that many entries after set 0 (else NULL, 0)
+    const ReplayCtl *rctl;   // replayable steps: reset flag and list length are read on the device (else NULL)
     long long d;             // elements per row
     long long cols_total;    // vector columns per row
     long long c_begin;       // first vector column handled by this launch
@@ -110,12 +109,11 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
     constexpr int UA = CSER_WALK_UA(MOM);                      // pass A: g (+ m)
     constexpr int UB = CSER_WALK_UB(RESET && ERR);             // pass B: x (+ e on reset steps)
     constexpr int UF = CSER_WALK_UF;                           // last pass: x only
-    const uint32_t rcur = P.rctl ? P.rctl->cur : 0u;
-    const uint8_t *__restrict__ mask_g = P.mask_g + (size_t)rcur * P.sel_stride;
-    const uint8_t *__restrict__ mask_r = P.mask_r + (size_t)rcur * P.sel_stride;
-    const uint32_t *__restrict__ list = P.list + (size_t)rcur * P.sel_stride;
-    const uint32_t n_listed = DENSE ? 0u : (P.rctl ? P.rctl->c[rcur].count : *P.count);
-    const bool reset_on = RESET && (P.rctl ? P.rctl->c[rcur].reset != 0 : true);
+    const uint8_t *__restrict__ mask_g = P.mask_g;
+    const uint8_t *__restrict__ mask_r = P.mask_r;
+    const uint32_t *__restrict__ list = P.list;
+    const uint32_t n_listed = DENSE ? 0u : (P.rctl ? P.rctl->c[0].count : *P.count);
+    const bool reset_on = RESET && (P.rctl ? P.rctl->c[0].reset != 0 : true);
     const unsigned long long total =
         DENSE ? (unsigned long long)(P.c_end - P.c_begin) : (unsigned long long)n_listed * P.bsv;
     const long long d = P.d;
@@ -310,11 +308,8 @@ __global__ void __launch_bounds__(kStepThreads, 8) cser_stream_kernel(const Step
     if (c >= P.c_end) return;
     const long long b = (P.c_end <= 0xffffffffll) ? (long long)((uint32_t)c / P.bsv)
                                                   : (long long)((unsigned long long)c / P.bsv);
-    const uint32_t rcur = P.rctl ? P.rctl->cur : 0u;
-    if (P.mask_g[(size_t)rcur * P.sel_stride + b] != 0) return;
-    if (RESET && P.mask_r[(size_t)rcur * P.sel_stride + b] != 0 &&
-        (P.rctl == nullptr || P.rctl->c[rcur].reset != 0))
-        return;
+    if (P.mask_g[b] != 0) return;
+    if (RESET && P.mask_r[b] != 0 && (P.rctl == nullptr || P.rctl->c[0].reset != 0)) return;
     // C(p) = 0, so p' = r = p (Algorithm 3 lines 4-8): x_i -= p_i, e_i -= p_i (no e array in
     // implementation II).
     const long long o = (long long)row * P.d + c * V;
