@@ -34,6 +34,7 @@ NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2_wrn40x8_n8_R32_H8": 1.7983e9 * 35_748_708 
 NO_ERROR_ARRAY = False   # --impl2: implementation II of Appendix A.4 (no e array)
 EXACT_COUNT = False      # --exact-count: every mask selects exactly round(B/R) blocks
 L2_RESIDENT = False      # ask the library to keep a small state in L2 (CSER_FLAG_L2_RESIDENT)
+STAGED = False           # --staged: selected blocks through the shared-memory staged kernel (CSER_FLAG_STAGED_SELECTED)
 
 
 def algorithmic_bytes(w, frac_e_touched):
@@ -257,7 +258,7 @@ def run_workload(w, K, W, dev, rank, world, ring_n=0, with_e2e=True, flush_l2=Fa
     opt = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
                  block_begin=0 if EXACT_COUNT else rank * w.n_blocks,
                  flags=(b.FLAG_NO_ERROR_ARRAY if NO_ERROR_ARRAY else 0) | (b.FLAG_EXACT_COUNT if EXACT_COUNT else 0)
-                 | (b.FLAG_L2_RESIDENT if L2_RESIDENT else 0))
+                 | (b.FLAG_L2_RESIDENT if L2_RESIDENT else 0) | (b.FLAG_STAGED_SELECTED if STAGED else 0))
     opt.set_x0(synth.x0(w, dev))
     g_bytes = w.n_workers * w.d * 4
     ring_n = ring_n or max(2, min(4, int(6e9 // g_bytes)))
@@ -427,18 +428,30 @@ def main():
     ap.add_argument("--d", type=int, default=0, help="override the vector length (small profiling cases)")
     ap.add_argument("--impl2", action="store_true", help="implementation II (no error array) as the main run")
     ap.add_argument("--exact-count", action="store_true", help="exact-count GRBS masks as the main run")
+    ap.add_argument("--R1", type=int, default=-1, help="override the update compressor's ratio")
+    ap.add_argument("--R2", type=int, default=-1, help="override the reset compressor's ratio")
+    ap.add_argument("--H", type=int, default=-1, help="override the reset interval")
+    ap.add_argument("--staged", action="store_true",
+                    help="selected blocks through the shared-memory staged kernel instead of the register-walking one")
+    ap.add_argument("--flush-l2", action="store_true", help="per-kernel figures with L2 flushed between launches")
     ap.add_argument("--oracle-slab", type=int, default=-1, help=argparse.SUPPRESS)
     ap.add_argument("--oracle-seconds", type=float, default=10.0, help=argparse.SUPPRESS)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
-    global NO_ERROR_ARRAY, EXACT_COUNT
+    global NO_ERROR_ARRAY, EXACT_COUNT, STAGED
     NO_ERROR_ARRAY = bool(args.impl2)
     EXACT_COUNT = bool(args.exact_count)
+    STAGED = bool(args.staged)
 
     from paper_2007_13221_b200 import synth
     w = synth.CONFIGS[args.config]
     if args.d:
         w = w.scaled(args.d)
+    if args.R1 >= 0 or args.R2 >= 0 or args.H >= 0:
+        from dataclasses import replace
+        w = replace(w, R1=args.R1 if args.R1 >= 0 else w.R1, R2=args.R2 if args.R2 >= 0 else w.R2,
+                    H=args.H if args.H >= 0 else w.H)
+        w = replace(w, name=f"{w.name}@R1={w.R1},R2={w.R2},H={w.H}")
     if args.oracle_slab >= 0:
         oracle_slab_worker(w, args.oracle_slab, args.oracle_seconds)
         return
@@ -465,14 +478,15 @@ def main():
         dist.barrier()
 
     K, W = args.steps, args.warmup
-    r = run_workload(w, K, W, dev, rank, world, ring_n=args.ring, with_e2e=not args.no_e2e)
+    r = run_workload(w, K, W, dev, rank, world, ring_n=args.ring, with_e2e=not args.no_e2e,
+                     flush_l2=args.flush_l2)
     alg_bytes = r["alg_bytes"]
 
     # the other workloads and variants, briefly (single GPU, default invocation only); a failure
     # here is recorded and never costs the headline line
     others = None
     if world == 1 and args.config == 2 and not args.d and not args.no_others and not args.impl2 \
-            and not args.exact_count:
+            and not args.exact_count and not args.staged and w is synth.CONFIGS[2]:
         others = {}
 
         def guarded(name, fn):

@@ -44,7 +44,11 @@
  *
  * Errors.  Functions returning int give 0 on success or a negative code below;
  * cser_last_error() returns a thread-local message for the last failure.  No call
- * aborts, throws, or traps on the device.
+ * aborts, throws, or traps on the device.  The only device-side waits are those of the
+ * opt-in kernel of CSER_FLAG_STAGED_SELECTED (a kernel waiting for its own asynchronous
+ * copies into shared memory); they are bounded to about a second, and one that ran out
+ * raises a host-visible word in the handle: every later cser_step / cser_read_state on
+ * that handle then returns CSER_ERR_CUDA, the step it happened in being incomplete.
  */
 #ifndef CSER_H_
 #define CSER_H_
@@ -132,6 +136,19 @@ cser_handle cser_create_slab(int64_t d, int32_t n_workers, int32_t block_size,
  *       destroyed, which is why it is opt-in.  Ignored when the state does not fit.
  */
 #define CSER_FLAG_L2_RESIDENT 4u
+/*
+ *   CSER_FLAG_STAGED_SELECTED  the blocks selected by a mask (Algorithm 3 line 7: the mean over
+ *       workers) are normally handled by a kernel in which a thread walks the worker axis of its
+ *       column with a few loads held in registers.  With this flag they go through an alternative
+ *       kernel instead, which brings all workers' segments of a block into shared memory with
+ *       asynchronous bulk copies (a producer warp, a ring of stages, shared-memory barriers with
+ *       bounded waits) and reduces from there.  Results are bit-identical.  On B200 the alternative is
+ *       slower at every ratio that was measured, which is why it is opt-in; it is kept so that the
+ *       comparison can be repeated.  It needs d and block_size to be multiples of 4, blocks of at
+ *       least 64 elements and few enough workers for one stage of shared memory; otherwise the flag
+ *       has no effect.
+ */
+#define CSER_FLAG_STAGED_SELECTED 8u
 cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size,
                            uint32_t R1, uint32_t R2, int32_t H,
                            float eta, float beta, uint64_t seed, int64_t block_begin,
@@ -291,12 +308,17 @@ int64_t cser_launch_count(cser_handle h);
  * CSER_ERR_INVALID; choose a larger block_size or use the handle API.
  *
  * The first call on each device looks up the array's device address (no allocation,
- * but a runtime query); make that first call outside any stream capture.
+ * but a runtime query); make that first call outside any stream capture.  As with
+ * cser_step, t and the rotation of the list counters are launch arguments, so a stream
+ * capture of the call must not be replayed.
  * All calls on a device share the one array: the masks and list of a call are
  * overwritten by the next.  Each call rewrites every entry it later reads and clears the
  * list counter the following call will use, so no clearing is needed between calls, but
  * two calls whose kernels may overlap on the GPU (different streams, or different host
- * threads) race on the array - serialize them on one stream and one host thread.
+ * threads) race on the array - serialize them on one stream and one host thread.  (Such
+ * a race gives wrong masks, hence a wrong step; it cannot write outside the array or
+ * outside the caller's arrays: list appends and list reads are bounded by the number of
+ * blocks.)
  * No cudaMalloc, cudaFree or other allocating routine is called.
  */
 #define CSER_NOALLOC_MAX_BLOCKS 262144

@@ -48,6 +48,7 @@ int fail(int code, const char *fmt, ...) {
 
 #include "grbs_kernels.cuh"
 #include "step_kernels.cuh"
+#include "staged_kernel.cuh"
 #include "wshard_kernels.cuh"
 
 }  // namespace
@@ -71,6 +72,9 @@ struct cser_ctx {
     uint32_t *sel_list = nullptr;                    // [B] blocks selected this step
     const uint32_t *cur_count = nullptr;             // how many
     uint8_t *last_mask_r = nullptr;                  // reset mask of the last reset step
+    // The reset mask of reset number q = t / H lives in half q & 1 of the reset-mask allocation, so the
+    // select kernel that prepares the next reset step never overwrites the last reset step's mask.
+    uint8_t *mask_r_half[2] = {nullptr, nullptr};
     // The masks of an iteration depend only on (seed, t), so the select kernel of iteration
     // t + 1 runs during iteration t, beside the step kernels, into the other buffer set.
     struct SelBuf {
@@ -100,7 +104,16 @@ struct cser_ctx {
     // auxiliary stream they run side by side (fork after the select kernel, join after both).
     cudaStream_t aux = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
-    const float *last_grad_checked = nullptr;        // last gradient pointer verified to be device memory
+    // The prefetched select kernel runs on aux behind the join, off the caller's stream; whoever next
+    // touches the buffer sets waits for ev_pre first.
+    cudaEvent_t ev_pre = nullptr;
+    bool pre_pending = false;
+    // Shared-memory staged selected-block kernel (CSER_FLAG_STAGED_SELECTED), 128-bit path only.
+    // Its bounded waits report through err_host, one word of mapped pinned host memory that the host
+    // looks at on every call without synchronizing.
+    bool staging = false;
+    int sm_count = 0;
+    unsigned *err_host = nullptr, *err_dev = nullptr;
     float *x0_stage = nullptr;                       // [d] staging for a host x0
     bool masks_injected = false;
     bool vec4 = false;                               // 128-bit path usable for the state arrays
@@ -124,6 +137,21 @@ uint32_t exact_k(long long B, uint32_t R) {
     if (R == 0) return 0;
     const long long k = (2 * B + R) / (2 * (long long)R);
     return (uint32_t)(k > B ? B : k);
+}
+
+// Where the reset mask of iteration t is kept (t a reset step).
+uint8_t *reset_mask_of(const cser_ctx *h, uint64_t t) {
+    if (h->n_buf != 2 || !h->mask_r_half[0]) return h->sb[0].mask_r;
+    return h->mask_r_half[(t / (uint64_t)h->H) & 1u];
+}
+
+// Order stream s behind a select kernel that is still running ahead on the auxiliary stream.
+int join_prefetch(cser_ctx *h, cudaStream_t s) {
+    if (h->pre_pending) {
+        CU_TRY(cudaStreamWaitEvent(s, h->ev_pre, 0));
+        h->pre_pending = false;
+    }
+    return CSER_OK;
 }
 
 // Select kernel(s) of iteration `t` into buffer set `buf`, on stream s.  Counter k % 3 is
@@ -156,7 +184,7 @@ int launch_select(cser_ctx *h, int buf, uint64_t t, bool is_reset, bool draw, cu
             CU_TRY(cudaGetLastError());
         }
     }
-    grbs_select_kernel<<<grid, 256, 0, s>>>(h->sb[buf].mask_g, h->sb[buf].mask_r, h->sb[buf].list, count,
+    grbs_select_kernel<<<grid, 256, 0, s>>>(h->sb[buf].mask_g, reset_mask_of(h, t), h->sb[buf].list, count,
                                             count_next, h->B, h->block_begin, k0, k1, t_lo, t_hi, R_g, R_r,
                                             is_reset ? 1 : 0, draw ? 1 : 0,
                                             h->exact_scratch ? h->exact_scratch->thr : nullptr, exact_g, exact_r);
@@ -168,18 +196,19 @@ int launch_select(cser_ctx *h, int buf, uint64_t t, bool is_reset, bool draw, cu
 }
 
 // Make buffer set `buf` (with its list counter) the current step's.
-void activate_selection(cser_ctx *h, int buf, const uint32_t *count, bool is_reset) {
+void activate_selection(cser_ctx *h, int buf, const uint32_t *count, bool is_reset, uint64_t t) {
     h->cur = buf;
-    h->mask_g = h->sb[buf].mask_g, h->mask_r = h->sb[buf].mask_r, h->sel_list = h->sb[buf].list;
+    h->mask_g = h->sb[buf].mask_g, h->sel_list = h->sb[buf].list;
     h->cur_count = count;
-    if (is_reset) h->last_mask_r = h->sb[buf].mask_r;
+    if (is_reset) h->mask_r = h->last_mask_r = reset_mask_of(h, t);
 }
 
 // Masks and list for iteration h->t: take the prefetched ones if they are for this iteration,
 // else run the select kernel now on stream s.
 int select_for_iteration(cser_ctx *h, bool is_reset, cudaStream_t s) {
+    if (int rc = join_prefetch(h, s)) return rc;
     if (h->pre_valid && h->pre_t == h->t && !h->masks_injected) {
-        activate_selection(h, h->cur ^ 1, h->pre_count, is_reset);
+        activate_selection(h, h->cur ^ 1, h->pre_count, is_reset, h->t);
         h->pre_valid = false;
         h->walk_all = false;
         return CSER_OK;
@@ -187,11 +216,62 @@ int select_for_iteration(cser_ctx *h, bool is_reset, cudaStream_t s) {
     const int nb = h->n_buf == 2 ? (h->cur ^ 1) : 0;
     const uint32_t *count = nullptr;
     if (int rc = launch_select(h, nb, h->t, is_reset, !h->masks_injected, s, &count)) return rc;
-    activate_selection(h, nb, count, is_reset);
+    activate_selection(h, nb, count, is_reset, h->t);
     h->pre_valid = false;
     h->walk_all = h->masks_injected;
     h->masks_injected = false;
     return CSER_OK;
+}
+
+// Work-unit geometry of the staged selected-block kernel: C vector columns per unit so that all n
+// workers' segments of every array fit one stage, blocks cut into equal chunks, as many stages as fit
+// the CTA's shared-memory budget.
+struct StagedGeom {
+    unsigned C = 0, n_chunks = 0, stages = 0;
+    size_t smem = 0;
+    bool ok = false;
+};
+
+StagedGeom staged_geometry(int n, unsigned bsv, bool mom, bool reset_err) {
+    StagedGeom G;
+    const unsigned long long per_col = (2ull + (mom ? 1 : 0) + (reset_err ? 1 : 0)) * (unsigned long long)n * 16ull;
+    unsigned long long cmax = kStagedStageBudget / per_col;
+    if (cmax > bsv) cmax = bsv;
+    if (cmax > kStagedMaxChunkCols) cmax = kStagedMaxChunkCols;
+    if (cmax < kStagedMinChunkCols) return G;          // too many workers or tiny blocks: register walk
+    if (cmax < bsv) cmax = cmax / 8 * 8;
+    unsigned chunks = (unsigned)((bsv + cmax - 1) / cmax);
+    unsigned C = (bsv + chunks - 1) / chunks;
+    if (chunks > 1) C = (C + 7) / 8 * 8;
+    chunks = (bsv + C - 1) / C;
+    const size_t stage = (size_t)per_col * C;
+    size_t stages = (kStagedCtaBudget - kStagedCtlBytes) / stage;
+    if (stages > (size_t)kStagedMaxStages) stages = kStagedMaxStages;
+    if (stages < 2) return G;
+    G.C = C, G.n_chunks = chunks, G.stages = (unsigned)stages;
+    G.smem = kStagedCtlBytes + stages * stage;
+    G.ok = true;
+    return G;
+}
+
+template <bool MOM, bool RESET, bool ERR, bool DENSE>
+cudaError_t launch_staged(int device, const StepParams &Q, unsigned grid, size_t smem, cudaStream_t st,
+                          cudaLaunchAttribute *attr, int n_attr) {
+    static bool configured[64] = {};
+    auto kernel = cser_selected_staged_kernel<MOM, RESET, ERR, DENSE>;
+    if (device < 0 || device >= 64 || !configured[device]) {
+        cudaError_t er = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)kStagedCtaBudget);
+        if (er != cudaSuccess) return er;
+#ifdef CSER_STAGED_CARVEOUT
+        cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, CSER_STAGED_CARVEOUT);
+#endif
+        if (device >= 0 && device < 64) configured[device] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid), cfg.blockDim = dim3(kStagedThreads), cfg.dynamicSmemBytes = smem, cfg.stream = st;
+    cfg.attrs = attr, cfg.numAttrs = n_attr;
+    return cudaLaunchKernelEx(&cfg, kernel, Q);
 }
 
 template <int V>
@@ -200,14 +280,15 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     const long long cols = P.c_end - P.c_begin;
     if (cols <= 0) return CSER_OK;
     const long long tiles = (cols + kStepThreads - 1) / kStepThreads;
-    const long long grid_ll = tiles * P.n;
-    if (grid_ll > 0x7fffffffll) return fail(CSER_ERR_INVALID, "n_workers * d too large for one launch");
+    if (tiles > 0x7fffffffll) return fail(CSER_ERR_INVALID, "d too large for one launch");
+    // The streaming kernel's grid is tiles x workers; more CTAs than one grid holds are launched in
+    // groups of whole rows.
+    const int rows_per_launch = (int)((0x7fffffffll / tiles) < (long long)P.n ? (0x7fffffffll / tiles) : P.n);
     StepParams Q = P;
     Q.tiles = (unsigned)tiles;
     Q.rctl = h->replay ? h->ctl : nullptr;
     if (h->replay) Q.mask_g = h->sb[0].mask_g, Q.mask_r = h->sb[0].mask_r, Q.list = h->sb[0].list;
     if (h->replay) is_reset = true;   // the reset variants decide on the device whether this step resets
-    const unsigned grid = (unsigned)grid_ll;
     // Grid of the selected-block kernel: the count lives on the device, so size the grid for
     // the expected number of selected columns in this launch's range plus slack; the kernel
     // strides over whatever the list really holds, so any grid size is correct.
@@ -221,31 +302,16 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     const bool mom = h->m != nullptr;
     // R1 == 1 selects every block on every step: nothing is left to stream.
     const bool stream_any = h->walk_all || h->R1 != 1;
-    cudaStream_t ws = s;
-    const bool fork = use_aux && h->aux != nullptr && stream_any;
-    const bool prefetch = !h->replay && h->n_buf == 2;
+    const bool have_aux = use_aux && h->aux != nullptr && h->n_total == 0;
+    const bool beside = have_aux && stream_any;                       // selected-block kernel beside the streaming one
+    const bool prefetch = have_aux && !h->replay && h->n_buf == 2;    // next iteration's select kernel on aux
+    const bool fork = beside || prefetch;
     if (fork) {
         CU_TRY(cudaEventRecord(h->ev_fork, s));
         CU_TRY(cudaStreamWaitEvent(h->aux, h->ev_fork, 0));
-        ws = h->aux;
     }
+    cudaStream_t ws = beside ? h->aux : s;
     const bool err = h->e != nullptr;
-    if (h->n_total > 0) {
-        // worker-sharded: the selected blocks go through pack / all-reduce / apply; only stream here
-        const bool mom_ = h->m != nullptr;
-        if (mom_) {
-            if (is_reset) cser_stream_kernel<V, true, true, true><<<grid, kStepThreads, 0, s>>>(Q);
-            else          cser_stream_kernel<V, true, false, true><<<grid, kStepThreads, 0, s>>>(Q);
-        } else {
-            if (is_reset) cser_stream_kernel<V, false, true, true><<<grid, kStepThreads, 0, s>>>(Q);
-            else          cser_stream_kernel<V, false, false, true><<<grid, kStepThreads, 0, s>>>(Q);
-        }
-        h->launches++;
-        CU_TRY(cudaGetLastError());
-        return CSER_OK;
-    }
-    const bool dense = frac >= kDenseWalkFraction;
-    if (dense) wgrid = wmax;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeAccessPolicyWindow;
     attr[0].val.accessPolicyWindow.base_ptr = h->state_base;
@@ -253,21 +319,67 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     attr[0].val.accessPolicyWindow.hitRatio = 1.0f;
     attr[0].val.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
     attr[0].val.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
-    auto launch = [&](void (*kernel)(const StepParams), unsigned g, unsigned threads, cudaStream_t st) {
+    auto launch = [&](void (*kernel)(const StepParams), const StepParams &A, unsigned g, unsigned threads,
+                      cudaStream_t st) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(g), cfg.blockDim = dim3(threads), cfg.dynamicSmemBytes = 0, cfg.stream = st;
         cfg.attrs = attr, cfg.numAttrs = h->l2_persist ? 1 : 0;
-        return cudaLaunchKernelEx(&cfg, kernel, Q);
+        return cudaLaunchKernelEx(&cfg, kernel, A);
     };
+    // streaming kernel: one launch per group of whole rows (one group unless tiles x workers > 2^31 - 1)
+    auto launch_stream = [&](void (*kernel)(const StepParams)) {
+        cudaError_t er = cudaSuccess;
+        for (int r0 = 0; r0 < P.n && er == cudaSuccess; r0 += rows_per_launch) {
+            const int rows = P.n - r0 < rows_per_launch ? P.n - r0 : rows_per_launch;
+            StepParams A = Q;
+            const long long off = (long long)r0 * P.d;
+            A.g += off, A.x += off;
+            if (A.e) A.e += off;
+            if (A.m) A.m += off;
+            er = launch(kernel, A, (unsigned)(tiles * rows), kStepThreads, s);
+            h->launches++;
+        }
+        return er;
+    };
+    if (h->n_total > 0) {
+        // worker-sharded: the selected blocks go through pack / all-reduce / apply; only stream here
+        cudaError_t er;
+        if (mom) er = is_reset ? launch_stream(cser_stream_kernel<V, true, true, true>)
+                               : launch_stream(cser_stream_kernel<V, true, false, true>);
+        else     er = is_reset ? launch_stream(cser_stream_kernel<V, false, true, true>)
+                               : launch_stream(cser_stream_kernel<V, false, false, true>);
+        CU_TRY(er);
+        CU_TRY(cudaGetLastError());
+        return CSER_OK;
+    }
+    const bool dense = frac >= kDenseWalkFraction;
+    if (dense) wgrid = wmax;
+    // The staged kernel (128-bit path only): persistent CTAs, two per SM, over the work units.
+    StagedGeom G;
+    if (V == 4 && h->staging) G = staged_geometry(P.n, P.bsv, mom, is_reset && err);
+    unsigned sgrid = 1;
+    if (G.ok) {
+        Q.chunk_cols = G.C, Q.n_chunks = G.n_chunks, Q.stages = G.stages, Q.err_word = h->err_dev;
+        const double entries = dense ? (double)cols / P.bsv + 2.0 : blocks;
+        const double units = entries * G.n_chunks;
+        const double cap = (double)kStagedCtasPerSm * (h->sm_count > 0 ? h->sm_count : 148);
+        sgrid = (unsigned)(units < cap ? (units < 1.0 ? 1.0 : units) : cap);
+    }
     cudaError_t lerr = cudaSuccess;
 #define CSER_LAUNCH_PAIR(MOM_, RESET_, ERR_)                                                            \
     do {                                                                                                \
-        if (dense)                                                                                      \
-            lerr = launch(cser_selected_kernel<V, MOM_, RESET_, ERR_, true>, (unsigned)wgrid, kWalkThreads, ws); \
+        if (G.ok && dense)                                                                              \
+            lerr = launch_staged<MOM_, RESET_, ERR_, true>(h->device, Q, sgrid, G.smem, ws, attr,       \
+                                                           h->l2_persist ? 1 : 0);                      \
+        else if (G.ok)                                                                                  \
+            lerr = launch_staged<MOM_, RESET_, ERR_, false>(h->device, Q, sgrid, G.smem, ws, attr,      \
+                                                            h->l2_persist ? 1 : 0);                     \
+        else if (dense)                                                                                 \
+            lerr = launch(cser_selected_kernel<V, MOM_, RESET_, ERR_, true>, Q, (unsigned)wgrid, kWalkThreads, ws); \
         else                                                                                            \
-            lerr = launch(cser_selected_kernel<V, MOM_, RESET_, ERR_, false>, (unsigned)wgrid, kWalkThreads, ws); \
+            lerr = launch(cser_selected_kernel<V, MOM_, RESET_, ERR_, false>, Q, (unsigned)wgrid, kWalkThreads, ws); \
         if (stream_any && lerr == cudaSuccess)                                                          \
-            lerr = launch(cser_stream_kernel<V, MOM_, RESET_, ERR_>, grid, kStepThreads, s);            \
+            lerr = launch_stream(cser_stream_kernel<V, MOM_, RESET_, ERR_>);                            \
     } while (0)
 #define CSER_LAUNCH_ERR(MOM_, RESET_)                                                                   \
     do {                                                                                                \
@@ -283,7 +395,7 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     }
 #undef CSER_LAUNCH_ERR
 #undef CSER_LAUNCH_PAIR
-    h->launches += stream_any ? 2 : 1;
+    h->launches += 1;
     CU_TRY(lerr);
     CU_TRY(cudaGetLastError());
     if (h->replay) {
@@ -296,18 +408,21 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
         h->launches++;
         CU_TRY(cudaGetLastError());
     }
-    if (fork) {
-        int rc = CSER_OK;
-        if (prefetch) {
-            // next iteration's select kernel, off the critical path
-            const uint64_t t_next = h->t + 1;
-            rc = launch_select(h, h->cur ^ 1, t_next, (t_next % (uint64_t)h->H) == 0, true, h->aux,
-                               &h->pre_count);
-            h->pre_valid = rc == CSER_OK;
-            h->pre_t = t_next;
-        }
-        CU_TRY(cudaEventRecord(h->ev_join, h->aux));      // join even if the prefetch could not be launched
+    if (beside) {
+        // join: the caller's stream continues once the selected-block kernel is done ...
+        CU_TRY(cudaEventRecord(h->ev_join, h->aux));
         CU_TRY(cudaStreamWaitEvent(s, h->ev_join, 0));
+    }
+    if (prefetch) {
+        // ... while the next iteration's select kernel runs on the auxiliary stream, off the critical
+        // path; the next call that touches the buffer sets waits for ev_pre
+        const uint64_t t_next = h->t + 1;
+        const int rc = launch_select(h, h->cur ^ 1, t_next, (t_next % (uint64_t)h->H) == 0, true, h->aux,
+                                     &h->pre_count);
+        h->pre_valid = rc == CSER_OK;
+        h->pre_t = t_next;
+        CU_TRY(cudaEventRecord(h->ev_pre, h->aux));
+        h->pre_pending = true;
         return rc;
     }
     return CSER_OK;
@@ -321,6 +436,8 @@ int launch_step(cser_ctx *h, const float *grad, long long col0, long long col1, 
     P.mask_g = h->mask_g, P.mask_r = h->mask_r;
     P.list = h->sel_list, P.count = h->cur_count;
     P.tiles = 0, P.rctl = nullptr;
+    P.list_cap = (unsigned)h->B;
+    P.chunk_cols = P.n_chunks = P.stages = 0, P.err_word = nullptr;
     P.d = h->d, P.n = h->n;
     P.eta = h->eta, P.beta = h->beta, P.n_f = (float)h->n;
     const bool v4 = h->vec4 && ((uintptr_t)grad % 16 == 0) && (col0 % 4 == 0) &&
@@ -354,7 +471,34 @@ int check_device_ptr(const void *p, const char *what) {
     }
     if (a.type != cudaMemoryTypeDevice && a.type != cudaMemoryTypeManaged)
         return fail(CSER_ERR_INVALID, "%s must be device memory", what);
+    if (a.type == cudaMemoryTypeDevice) {
+        // memory of another GPU would be dereferenced by kernels of this one
+        int dev = -1;
+        if (cudaGetDevice(&dev) == cudaSuccess && a.device != dev)
+            return fail(CSER_ERR_INVALID, "%s lives on device %d, the current device is %d", what, a.device, dev);
+    }
     return CSER_OK;
+}
+
+// A bounded device-side wait that ran out (see staged_kernel.cuh) left its code in the handle's
+// host-visible word: every later call reports it instead of stepping on an incomplete state.
+int check_device_error(cser_ctx *h) {
+    if (h->err_host) {
+        const unsigned code = *reinterpret_cast<volatile unsigned *>(h->err_host);
+        if (code)
+            return fail(CSER_ERR_CUDA,
+                        "a device-side wait ran out in an earlier step (code 0x%x): that step is incomplete, "
+                        "restore the state from a checkpoint into a new handle", code);
+    }
+    return CSER_OK;
+}
+
+// An iteration whose launches could not all be enqueued did not happen: t goes back to where it was
+// and the prepared masks are dropped, so that a retry draws them again.
+int abandon_iteration(cser_ctx *h, uint64_t t_before, int rc) {
+    h->t = t_before;
+    h->pre_valid = false;
+    return rc;
 }
 
 // advance t and decide whether this iteration resets (Algorithm 2 line 8)
@@ -378,7 +522,8 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
         fail(CSER_ERR_INVALID, "cser_create: d, n_workers, block_size, R2, H must be positive");
         return nullptr;
     }
-    if (flags & ~(uint32_t)(CSER_FLAG_NO_ERROR_ARRAY | CSER_FLAG_EXACT_COUNT | CSER_FLAG_L2_RESIDENT)) {
+    if (flags & ~(uint32_t)(CSER_FLAG_NO_ERROR_ARRAY | CSER_FLAG_EXACT_COUNT | CSER_FLAG_L2_RESIDENT |
+                            CSER_FLAG_STAGED_SELECTED)) {
         fail(CSER_ERR_INVALID, "cser_create: unknown flags 0x%x", flags);
         return nullptr;
     }
@@ -427,6 +572,7 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
     if (er == cudaSuccess) {
         h->sb[1].mask_g = h->sb[0].mask_g + B, h->sb[1].mask_r = h->sb[0].mask_r + B;
         h->sb[1].list = h->sb[0].list + B;
+        h->mask_r_half[0] = h->sb[0].mask_r, h->mask_r_half[1] = h->sb[1].mask_r;
     }
     if (er == cudaSuccess) er = cudaMemset(h->state_base, 0, h->state_bytes);
     if (er == cudaSuccess && (flags & CSER_FLAG_L2_RESIDENT)) {
@@ -444,6 +590,15 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
             cudaGetLastError();
         }
     }
+    if (er == cudaSuccess) er = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
+    if (er == cudaSuccess && (flags & CSER_FLAG_STAGED_SELECTED)) {
+        er = cudaHostAlloc(reinterpret_cast<void **>(&h->err_host), 64, cudaHostAllocMapped | cudaHostAllocPortable);
+        if (er == cudaSuccess) {
+            *h->err_host = 0;
+            er = cudaHostGetDevicePointer(reinterpret_cast<void **>(&h->err_dev), h->err_host, 0);
+        }
+        h->staging = er == cudaSuccess;
+    }
     h->exact = (flags & CSER_FLAG_EXACT_COUNT) != 0;
     if (er == cudaSuccess && h->exact) er = cudaMalloc(&h->exact_scratch, sizeof(ExactScratch));
     if (er == cudaSuccess && h->exact) er = cudaMemset(h->exact_scratch, 0, sizeof(ExactScratch));
@@ -452,7 +607,7 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
     if (er == cudaSuccess) er = cudaMemset(h->ctl, 0, sizeof(ReplayCtl));
     if (er == cudaSuccess) er = cudaMalloc(&h->sel_count, 3 * sizeof(uint32_t));
     if (er == cudaSuccess) er = cudaMemset(h->sel_count, 0, 3 * sizeof(uint32_t));
-    if (er == cudaSuccess) activate_selection(h, 0, h->sel_count, true);
+    if (er == cudaSuccess) activate_selection(h, 0, h->sel_count, true, 0);
     for (int k = 0; k < 3 && er == cudaSuccess; ++k) er = cudaEventCreate(&h->ev[k]);
     if (er == cudaSuccess) {
         int lo = 0, hi = 0;   // hi = numerically lowest = highest priority
@@ -461,6 +616,7 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
     }
     if (er == cudaSuccess) er = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
     if (er == cudaSuccess) er = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
+    if (er == cudaSuccess) er = cudaEventCreateWithFlags(&h->ev_pre, cudaEventDisableTiming);
     if (er == cudaSuccess) er = cudaDeviceSynchronize();
     if (er != cudaSuccess) {
         fail(er == cudaErrorMemoryAllocation ? CSER_ERR_NOMEM : CSER_ERR_CUDA, "cser_create: %s",
@@ -485,6 +641,7 @@ cser_handle cser_create(int64_t d, int32_t n_workers, int32_t block_size, uint32
 
 void cser_destroy(cser_handle h) {
     if (!h) return;
+    if (h->aux) cudaStreamSynchronize(h->aux);   // a select kernel may still be running ahead
     if (h->l2_persist) {
         cudaCtxResetPersistingL2Cache();
         cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, h->l2_limit_before);
@@ -493,6 +650,7 @@ void cser_destroy(cser_handle h) {
     cudaFree(h->state_base);
     cudaFree(h->sb[0].mask_g), cudaFree(h->sb[0].mask_r), cudaFree(h->sb[0].list);
     cudaFree(h->x0_stage), cudaFree(h->g_stage);
+    if (h->err_host) cudaFreeHost(h->err_host);
     cudaFree(h->sel_count), cudaFree(h->exact_scratch), cudaFree(h->exact_words), cudaFree(h->ctl);
     cudaFree(h->pos_g), cudaFree(h->pos_r), cudaFree(h->olist_g), cudaFree(h->olist_r);
     for (auto &ev : h->ev) if (ev) cudaEventDestroy(ev);
@@ -501,6 +659,7 @@ void cser_destroy(cser_handle h) {
     if (h->aux) cudaStreamDestroy(h->aux);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
+    if (h->ev_pre) cudaEventDestroy(h->ev_pre);
     delete h;
 }
 
@@ -530,19 +689,20 @@ int cser_set_x0(cser_handle h, const float *x0, void *stream) {
 
 int cser_step(cser_handle h, const float *grad, void *stream) {
     if (int rc = check_handle(h)) return rc;
-    if (!grad || grad != h->last_grad_checked) {   // the pointer query costs a microsecond: once per buffer
-        if (int rc = check_device_ptr(grad, "cser_step: grad")) return rc;
-        h->last_grad_checked = grad;
-    }
+    if (int rc = check_device_error(h)) return rc;
+    if (int rc = check_device_ptr(grad, "cser_step: grad")) return rc;   // every call: an address can be reused
     if ((uintptr_t)grad % 4 != 0) return fail(CSER_ERR_INVALID, "cser_step: grad is not 4-byte aligned");
     if (h->n_total > 0) return fail(CSER_ERR_INVALID, "cser_step: worker-sharded handle; use cser_wshard_pack/apply");
     if (h->replay) return fail(CSER_ERR_INVALID, "cser_step: between cser_replay_begin and cser_replay_end use cser_step_replayable");
     cudaStream_t s = (cudaStream_t)stream;
+    const uint64_t t_before = h->t;
     const bool is_reset = begin_iteration(h);
-    if (h->timing) CU_TRY(cudaEventRecord(h->ev[0], s));
-    if (int rc = select_for_iteration(h, is_reset, s)) return rc;
-    if (h->timing) CU_TRY(cudaEventRecord(h->ev[1], s));
-    if (int rc = launch_step(h, grad, 0, h->d, is_reset, s, true)) return rc;
+    int rc = CSER_OK;
+    if (h->timing && cudaEventRecord(h->ev[0], s) != cudaSuccess) rc = fail(CSER_ERR_CUDA, "cser_step: event record failed");
+    if (!rc) rc = select_for_iteration(h, is_reset, s);
+    if (!rc && h->timing && cudaEventRecord(h->ev[1], s) != cudaSuccess) rc = fail(CSER_ERR_CUDA, "cser_step: event record failed");
+    if (!rc) rc = launch_step(h, grad, 0, h->d, is_reset, s, true);
+    if (rc) return abandon_iteration(h, t_before, rc);
     if (h->timing) {
         CU_TRY(cudaEventRecord(h->ev[2], s));
         h->ev_valid = true;
@@ -552,6 +712,7 @@ int cser_step(cser_handle h, const float *grad, void *stream) {
 
 int cser_step_host(cser_handle h, const float *grad_host, void *stream) {
     if (int rc = check_handle(h)) return rc;
+    if (int rc = check_device_error(h)) return rc;
     if (!grad_host) return fail(CSER_ERR_INVALID, "cser_step_host: grad_host is NULL");
     if (h->n_total > 0) return fail(CSER_ERR_INVALID, "cser_step_host: worker-sharded handle");
     if (h->replay) return fail(CSER_ERR_INVALID, "cser_step_host: call cser_replay_end first");
@@ -561,9 +722,10 @@ int cser_step_host(cser_handle h, const float *grad_host, void *stream) {
         for (auto &st_ : h->hs) CU_TRY(cudaStreamCreateWithFlags(&st_, cudaStreamNonBlocking));
         for (auto &ev : h->h_ev) CU_TRY(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
     }
+    const uint64_t t_before = h->t;
     const bool is_reset = begin_iteration(h);
     // masks first, on the caller's stream; both internal streams start after them
-    if (int rc = select_for_iteration(h, is_reset, s)) return rc;
+    if (int rc = select_for_iteration(h, is_reset, s)) return abandon_iteration(h, t_before, rc);
     CU_TRY(cudaEventRecord(h->h_ev[0], s));
     CU_TRY(cudaStreamWaitEvent(h->hs[0], h->h_ev[0], 0));
     CU_TRY(cudaStreamWaitEvent(h->hs[1], h->h_ev[0], 0));
@@ -580,7 +742,7 @@ int cser_step_host(cser_handle h, const float *grad_host, void *stream) {
         CU_TRY(cudaMemcpy2DAsync(h->g_stage + c0, (size_t)d * sizeof(float), grad_host + c0,
                                  (size_t)d * sizeof(float), (size_t)(c1 - c0) * sizeof(float),
                                  (size_t)h->n, cudaMemcpyHostToDevice, cs));
-        if (int rc = launch_step(h, h->g_stage, c0, c1, is_reset, cs)) return rc;
+        if (int rc = launch_step(h, h->g_stage, c0, c1, is_reset, cs)) return abandon_iteration(h, t_before, rc);
     }
     CU_TRY(cudaEventRecord(h->h_ev[1], h->hs[0]));
     CU_TRY(cudaEventRecord(h->h_ev[2], h->hs[1]));
@@ -609,6 +771,7 @@ static int state_piece(cser_ctx *h, int which, void **ptr, size_t *bytes) {
 
 int cser_read_state(cser_handle h, int which, void *dst, size_t dst_bytes, void *stream) {
     if (int rc = check_handle(h)) return rc;
+    if (int rc = check_device_error(h)) return rc;
     if (!dst) return fail(CSER_ERR_INVALID, "cser_read_state: dst is NULL");
     void *src;
     size_t bytes;
@@ -687,9 +850,11 @@ int cser_debug_set_masks(cser_handle h, const uint8_t *g_mask, const uint8_t *r_
     if (next_is_reset && !r_mask)
         return fail(CSER_ERR_INVALID, "cser_debug_set_masks: next step resets, r_mask is NULL");
     cudaStream_t s = (cudaStream_t)stream;
+    if (int rc = join_prefetch(h, s)) return rc;
     const int nb = h->n_buf == 2 ? (h->cur ^ 1) : 0;   // the set the next step's select kernel reads
     CU_TRY(cudaMemcpyAsync(h->sb[nb].mask_g, g_mask, (size_t)h->B, cudaMemcpyDefault, s));
-    if (r_mask) CU_TRY(cudaMemcpyAsync(h->sb[nb].mask_r, r_mask, (size_t)h->B, cudaMemcpyDefault, s));
+    if (r_mask && next_is_reset)
+        CU_TRY(cudaMemcpyAsync(reset_mask_of(h, h->t + 1), r_mask, (size_t)h->B, cudaMemcpyDefault, s));
     h->masks_injected = true;
     return CSER_OK;
 }
@@ -791,8 +956,9 @@ int cser_wshard_pack(cser_handle h, const float *grad, float *msg, size_t msg_el
     if ((int64_t)msg_elems < cser_wshard_message_elems(h, next_reset))
         return fail(CSER_ERR_TOO_SMALL, "cser_wshard_pack: message buffer too small");
     cudaStream_t s = (cudaStream_t)stream;
+    const uint64_t t_before = h->t;
     const bool is_reset = begin_iteration(h);
-    if (int rc = select_for_iteration(h, is_reset, s)) return rc;
+    if (int rc = select_for_iteration(h, is_reset, s)) return abandon_iteration(h, t_before, rc);
     ordered_lists_kernel<<<1, 1024, 0, s>>>(h->mask_g, h->mask_r, h->B, is_reset ? 1 : 0, h->pos_g, h->pos_r,
                                             h->olist_g, h->olist_r);
     h->launches++;
@@ -830,6 +996,13 @@ int cser_replay_begin(cser_handle h, void *stream) {
         return fail(CSER_ERR_INVALID,
                     "cser_replay_begin: not available with exact-count masks, worker sharding or injected masks");
     cudaStream_t s = (cudaStream_t)stream;
+    if (int rc = join_prefetch(h, s)) return rc;
+    // In replay mode half 0 of the reset-mask allocation always holds the last executed reset step's
+    // mask (the advance kernel copies a prepared mask over it only when its step resets).
+    if (h->last_mask_r && h->last_mask_r != h->sb[0].mask_r) {
+        CU_TRY(cudaMemcpyAsync(h->sb[0].mask_r, h->last_mask_r, (size_t)h->B, cudaMemcpyDeviceToDevice, s));
+        h->last_mask_r = h->sb[0].mask_r;
+    }
     ReplayCtl c = {};
     c.c[0].t = h->t;           // block 0 stands for the iteration already done
     CU_TRY(cudaMemcpyAsync(h->ctl, &c, sizeof(c), cudaMemcpyHostToDevice, s));
@@ -850,10 +1023,8 @@ int cser_replay_begin(cser_handle h, void *stream) {
 int cser_step_replayable(cser_handle h, const float *grad, void *stream) {
     if (int rc = check_handle(h)) return rc;
     if (!h->replay) return fail(CSER_ERR_INVALID, "cser_step_replayable: call cser_replay_begin first");
-    if (!grad || grad != h->last_grad_checked) {
-        if (int rc = check_device_ptr(grad, "cser_step_replayable: grad")) return rc;
-        h->last_grad_checked = grad;
-    }
+    if (int rc = check_device_error(h)) return rc;
+    if (int rc = check_device_ptr(grad, "cser_step_replayable: grad")) return rc;
     if ((uintptr_t)grad % 4 != 0) return fail(CSER_ERR_INVALID, "cser_step_replayable: grad is not 4-byte aligned");
     cudaStream_t s = (cudaStream_t)stream;
     // the iteration prepared during the last step becomes the current one
@@ -873,7 +1044,17 @@ int cser_replay_end(cser_handle h, void *stream) {
     h->t = c.c[0].t;
     h->replay = false;
     h->pre_valid = false;
-    activate_selection(h, 0, h->sel_count, c.c[0].reset != 0);   // set 0 holds the masks of the last iteration
+    // Set 0 holds the masks of the last iteration, half 0 the last executed reset mask.  Ordinary steps
+    // keep reset number q's mask in half q & 1: if the next reset step would write half 0, move the last
+    // mask to half 1 first so that it stays readable until then.
+    h->cur = 0;
+    h->mask_g = h->sb[0].mask_g, h->sel_list = h->sb[0].list, h->cur_count = h->sel_count;
+    h->mask_r = h->last_mask_r = h->sb[0].mask_r;
+    const uint64_t next_reset = (h->t / (uint64_t)h->H + 1) * (uint64_t)h->H;
+    if (reset_mask_of(h, next_reset) == h->sb[0].mask_r && h->mask_r_half[1]) {
+        CU_TRY(cudaMemcpy(h->mask_r_half[1], h->sb[0].mask_r, (size_t)h->B, cudaMemcpyDeviceToDevice));
+        h->mask_r = h->last_mask_r = h->mask_r_half[1];
+    }
     return CSER_OK;
 }
 

@@ -175,7 +175,10 @@ grbs_select_kernel(uint8_t *__restrict__ mask_g, uint8_t *__restrict__ mask_r,
     unsigned base = 0;
     if ((int)lane == leader) base = atomicAdd(count, (unsigned)__popc(ballot));
     base = __shfl_sync(0xffffffffu, base, leader);
-    if (need) list[base + __popc(ballot & ((1u << lane) - 1u))] = (uint32_t)b;
+    // The list holds B entries.  A counter that was not cleared (overlapping allocation-free steps
+    // race on it) must not carry an append past the end.
+    const unsigned at = base + __popc(ballot & ((1u << lane) - 1u));
+    if (need && at < (unsigned long long)B) list[at] = (uint32_t)b;
 }
 
 
@@ -254,7 +257,8 @@ grbs_select_replay_kernel(ReplayCtl *R, uint8_t *__restrict__ mask_g, uint8_t *_
         unsigned base = 0;
         if ((int)lane == leader) base = atomicAdd(&out->count, (unsigned)__popc(ballot));
         base = __shfl_sync(0xffffffffu, base, leader);
-        if (need) list[base + __popc(ballot & ((1u << lane) - 1u))] = (uint32_t)b;
+        const unsigned at = base + __popc(ballot & ((1u << lane) - 1u));
+        if (need && at < (unsigned long long)B) list[at] = (uint32_t)b;
     }
     __syncthreads();
     if (threadIdx.x == 0) {

@@ -54,6 +54,12 @@ struct StepParams {
     long long c_end;         // one past the last
     unsigned bsv;            // GRBS block size in vector columns
     unsigned tiles;          // tiles of 256 vector columns in [c_begin, c_end)
+    unsigned list_cap;       // entries the list can hold (blocks of the vector): bounds whatever *count says
+    // shared-memory staged selected-block kernel only:
+    unsigned chunk_cols;     // vector columns per work unit
+    unsigned n_chunks;       // work units per block
+    unsigned stages;         // stages of the copy ring
+    unsigned *err_word;      // host-visible word a wait that ran out raises (may be NULL)
     int n;
     float eta, beta, n_f;
 };
@@ -79,13 +85,13 @@ __device__ __forceinline__ Pack<V> get_p(const Pack<V> &g, Pack<V> &m, float eta
 constexpr int kStepThreads = 256;   // streaming kernel: one CTA = 256 vector columns of one row
 constexpr int kWalkThreads = 128;   // selected-block kernel
 constexpr int kWalkBatch = 4;       // workers whose loads a walking thread keeps in flight (worker-sharded pack)
-// Batch sizes of the selected-block kernel.  Measured on B200: 2, 4 and 8 are within 2 % of each
-// other on every workload (more loads in flight per thread cost registers, hence occupancy).
+// Batch sizes of the selected-block kernel: workers whose loads are in flight together in each pass.
+// Measured on B200: 2, 4 and 8 are within 2 % of each other where few blocks are selected; with many
+// selected blocks 8 loses to 4 (more loads in flight per thread cost registers, hence occupancy).
 #ifndef CSER_WALK_UA
-#define CSER_WALK_UA(mom) 4
-#define CSER_WALK_UB(reset_err) 4
-#define CSER_WALK_UF 4
-#define CSER_WALK_UR(mom) 2
+#define CSER_WALK_UA 4      // update-selected, first pass: g (+ m) (+ e when the block is reset too)
+#define CSER_WALK_UB 4      // update-selected, second pass: x (+ e)
+#define CSER_WALK_UR 2      // reset-selected only: g (+ m) + x + e
 #endif
 #ifndef CSER_DENSE_WALK_FRACTION
 #define CSER_DENSE_WALK_FRACTION 0.3
@@ -95,9 +101,12 @@ constexpr double kDenseWalkFraction = CSER_DENSE_WALK_FRACTION;   // expected se
 // Selected blocks (1/R of the data): the update needs the mean over workers, so here one
 // thread owns one vector column of a selected block and walks the worker axis.  Threads
 // are laid over the concatenation of the listed blocks, so CTAs are full whatever the
-// block size.  Each pass issues the loads of kWalkBatch workers before it consumes any of
+// block size.  Each pass issues the loads of a batch of workers before it consumes any of
 // them (the in-place stores would otherwise keep the compiler from hoisting the next
 // worker's loads), and sums in ascending worker order starting from worker 0's value.
+// An update-selected block takes two passes over the worker axis: the first forms the means
+// (p-bar and, if the block is reset-selected too, e-bar), the second writes x (and e) once; the e it
+// reads again was read a moment ago by the same thread and comes from cache.
 // This kernel has its own register budget; the streaming kernel stays at 32 registers.
 // DENSE = false: threads are laid over the listed blocks (few blocks selected).  DENSE =
 // true: one thread per column of the whole range, returning at once if no mask selects its
@@ -105,20 +114,23 @@ constexpr double kDenseWalkFraction = CSER_DENSE_WALK_FRACTION;   // expected se
 // their natural order is worth more than the idle threads cost.
 template <int V, bool MOM, bool RESET, bool ERR, bool DENSE>
 __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepParams P) {
-    // workers whose loads are in flight together: fewer arrays per worker allow more workers
-    constexpr int UA = CSER_WALK_UA(MOM);                      // pass A: g (+ m)
-    constexpr int UB = CSER_WALK_UB(RESET && ERR);             // pass B: x (+ e on reset steps)
-    constexpr int UF = CSER_WALK_UF;                           // last pass: x only
+    constexpr int UA = CSER_WALK_UA, UB = CSER_WALK_UB, UR = CSER_WALK_UR;
     const uint8_t *__restrict__ mask_g = P.mask_g;
     const uint8_t *__restrict__ mask_r = P.mask_r;
     const uint32_t *__restrict__ list = P.list;
-    const uint32_t n_listed = DENSE ? 0u : (P.rctl ? P.rctl->c[0].count : *P.count);
+    // never trust the counter beyond the list's capacity (a caller that lets two allocation-free
+    // steps overlap can leave a stale count behind)
+    const uint32_t n_counted = DENSE ? 0u : (P.rctl ? P.rctl->c[0].count : *P.count);
+    const uint32_t n_listed = n_counted < P.list_cap ? n_counted : P.list_cap;
     const bool reset_on = RESET && (P.rctl ? P.rctl->c[0].reset != 0 : true);
     const unsigned long long total =
         DENSE ? (unsigned long long)(P.c_end - P.c_begin) : (unsigned long long)n_listed * P.bsv;
     const long long d = P.d;
     const int n = P.n;
-    const float eta = P.eta, beta = P.beta;
+    const float eta = P.eta, beta = P.beta, n_f = P.n_f;
+    Pack<V> zero;
+#pragma unroll
+    for (int k = 0; k < V; ++k) zero.v[k] = 0.f;
     for (unsigned long long f = (unsigned long long)blockIdx.x * kWalkThreads + threadIdx.x; f < total;
          f += (unsigned long long)gridDim.x * kWalkThreads) {
         long long c;
@@ -142,25 +154,24 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
         float *__restrict__ x = P.x + c * V;
         float *__restrict__ e = ERR ? P.e + c * V : nullptr;
         float *__restrict__ m = MOM ? P.m + c * V : nullptr;
-        // With an error array: sum over workers of e_{t-1/2}.  Without one (implementation
-        // II): sum over workers of x_{t-1/2}.  Reset-selected blocks only.
-        Pack<V> sum_r;
-#pragma unroll
-        for (int k = 0; k < V; ++k) sum_r.v[k] = 0.f;
 
         if (sg) {
-            // Update-selected block: r = 0, p' = mean_k p_k.  Pass A forms the mean and updates m.
-            Pack<V> sum_p;
-#pragma unroll
-            for (int k = 0; k < V; ++k) sum_p.v[k] = 0.f;
+            // Update-selected block (Algorithm 3 with C(v) = v): r = 0, p' = mean_k p_k.  First pass:
+            // the mean of p, m updated; if the block is reset-selected too (with an error array) the
+            // mean of e as well, e being unchanged by this step's update.
+            Pack<V> sum_p = zero, sum_r = zero;
+            const bool with_e = RESET && ERR && sr;
             for (int i0 = 0; i0 < n; i0 += UA) {
-                Pack<V> gv[UA], mv[UA];
+                Pack<V> gv[UA], mv[UA], ev[UA];
 #pragma unroll
                 for (int u = 0; u < UA; ++u) {
                     if (i0 + u < n) {
                         const long long o = (long long)(i0 + u) * d;
                         gv[u] = ld_stream<V>(g + o);
                         if constexpr (MOM) mv[u] = ld<V>(m + o);
+                        if constexpr (RESET && ERR) {
+                            if (with_e) ev[u] = ld<V>(e + o);
+                        }
                     }
                 }
 #pragma unroll
@@ -169,17 +180,49 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
                         const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], eta, beta);
                         if constexpr (MOM) st<V>(m + (long long)(i0 + u) * d, mv[u]);
 #pragma unroll
-                        for (int k = 0; k < V; ++k)
+                        for (int k = 0; k < V; ++k) {
                             sum_p.v[k] = (i0 + u == 0) ? p.v[k] : sum_p.v[k] + p.v[k];
+                            if constexpr (RESET && ERR) {
+                                if (with_e) sum_r.v[k] = (i0 + u == 0) ? ev[u].v[k] : sum_r.v[k] + ev[u].v[k];
+                            }
+                        }
                     }
                 }
             }
-            Pack<V> pbar;
+            Pack<V> pbar, rbar = zero;
 #pragma unroll
-            for (int k = 0; k < V; ++k) pbar.v[k] = sum_p.v[k] / P.n_f;
-            // Pass B: x_i -= p-bar; e untouched.  If the block is reset-selected too: with an
-            // error array store (x_i - p-bar) - e_i, zero e and gather sum_k e_k; without one
-            // gather sum_k (x_k - p-bar) and store nothing yet.
+            for (int k = 0; k < V; ++k) pbar.v[k] = sum_p.v[k] / n_f;
+            if constexpr (RESET && !ERR) {
+                if (sr) {
+                    // implementation II (Appendix A.4): x_i = mean_k (x_k - p-bar); one more pass over x
+                    for (int i0 = 0; i0 < n; i0 += UB) {
+                        Pack<V> xv[UB];
+#pragma unroll
+                        for (int u = 0; u < UB; ++u)
+                            if (i0 + u < n) xv[u] = ld<V>(x + (long long)(i0 + u) * d);
+#pragma unroll
+                        for (int u = 0; u < UB; ++u) {
+                            if (i0 + u < n) {
+#pragma unroll
+                                for (int k = 0; k < V; ++k) {
+                                    const float xh = xv[u].v[k] - pbar.v[k];
+                                    sum_r.v[k] = (i0 + u == 0) ? xh : sum_r.v[k] + xh;
+                                }
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int k = 0; k < V; ++k) rbar.v[k] = sum_r.v[k] / n_f;
+                    for (int i = 0; i < n; ++i) st<V>(x + (long long)i * d, rbar);
+                    continue;
+                }
+            }
+            if constexpr (RESET && ERR) {
+#pragma unroll
+                for (int k = 0; k < V; ++k) rbar.v[k] = sum_r.v[k] / n_f;
+            }
+            // Second pass: x_i -= p-bar, e untouched; on a reset-selected block (Algorithm 2 lines
+            // 11-12) x_i = ((x_i - p-bar) - e_i) + e-bar and e_i = 0.
             for (int i0 = 0; i0 < n; i0 += UB) {
                 Pack<V> xv[UB], ev[UB];
 #pragma unroll
@@ -187,8 +230,8 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
                     if (i0 + u < n) {
                         const long long o = (long long)(i0 + u) * d;
                         xv[u] = ld<V>(x + o);
-                        if constexpr (ERR) {
-                            if (sr) ev[u] = ld<V>(e + o);
+                        if constexpr (RESET && ERR) {
+                            if (with_e) ev[u] = ld<V>(e + o);
                         }
                     }
                 }
@@ -198,37 +241,28 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
                         const long long o = (long long)(i0 + u) * d;
 #pragma unroll
                         for (int k = 0; k < V; ++k) xv[u].v[k] = xv[u].v[k] - pbar.v[k];
-                        if (sr) {
-                            if constexpr (ERR) {
-                                Pack<V> z;
+                        if constexpr (RESET && ERR) {
+                            if (with_e) {
 #pragma unroll
-                                for (int k = 0; k < V; ++k) {
-                                    sum_r.v[k] = (i0 + u == 0) ? ev[u].v[k] : sum_r.v[k] + ev[u].v[k];
-                                    xv[u].v[k] = xv[u].v[k] - ev[u].v[k];
-                                    z.v[k] = 0.f;
-                                }
-                                st<V>(e + o, z);
-                                st<V>(x + o, xv[u]);
-                            } else {
-#pragma unroll
-                                for (int k = 0; k < V; ++k)
-                                    sum_r.v[k] = (i0 + u == 0) ? xv[u].v[k] : sum_r.v[k] + xv[u].v[k];
+                                for (int k = 0; k < V; ++k) xv[u].v[k] = (xv[u].v[k] - ev[u].v[k]) + rbar.v[k];
+                                st<V>(e + o, zero);
                             }
-                        } else {
-                            st<V>(x + o, xv[u]);
                         }
+                        st<V>(x + o, xv[u]);
                     }
                 }
             }
-        } else {
+        } else if constexpr (RESET) {
             // Selected by the reset mask only: take the residual step (x_{t-1/2} = x - p,
             // e_{t-1/2} = e - p).  With an error array store x_{t-1/2} - e_{t-1/2}, zero e and
-            // gather sum_k e_{k,t-1/2}; without one gather sum_k x_{k,t-1/2}.
-            constexpr int U2 = CSER_WALK_UR(MOM);             // g, x, e (+ m)
-            for (int i0 = 0; i0 < n; i0 += U2) {
-                Pack<V> gv[U2], mv[U2], xv[U2], ev[U2];
+            // gather sum_k e_{k,t-1/2}; without one gather sum_k x_{k,t-1/2}.  (Forming the sum in
+            // a pass of its own and writing x once was measured and is slower here: it reads g, m
+            // and e twice, and these blocks are too few for the re-reads to stay in L1.)
+            Pack<V> sum_r = zero;
+            for (int i0 = 0; i0 < n; i0 += UR) {
+                Pack<V> gv[UR], mv[UR], xv[UR], ev[UR];
 #pragma unroll
-                for (int u = 0; u < U2; ++u) {
+                for (int u = 0; u < UR; ++u) {
                     if (i0 + u < n) {
                         const long long o = (long long)(i0 + u) * d;
                         gv[u] = ld_stream<V>(g + o);
@@ -238,23 +272,21 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
                     }
                 }
 #pragma unroll
-                for (int u = 0; u < U2; ++u) {
+                for (int u = 0; u < UR; ++u) {
                     if (i0 + u < n) {
                         const long long o = (long long)(i0 + u) * d;
                         const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], eta, beta);
                         if constexpr (MOM) st<V>(m + o, mv[u]);
                         if constexpr (ERR) {
-                            Pack<V> z;
 #pragma unroll
                             for (int k = 0; k < V; ++k) {
                                 const float xh = xv[u].v[k] - p.v[k];
                                 const float eh = ev[u].v[k] - p.v[k];
                                 sum_r.v[k] = (i0 + u == 0) ? eh : sum_r.v[k] + eh;
                                 xv[u].v[k] = xh - eh;
-                                z.v[k] = 0.f;
                             }
                             st<V>(x + o, xv[u]);
-                            st<V>(e + o, z);
+                            st<V>(e + o, zero);
                         } else {
 #pragma unroll
                             for (int k = 0; k < V; ++k) {
@@ -265,22 +297,19 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
                     }
                 }
             }
-        }
-
-        if (sr) {
             Pack<V> rbar;
 #pragma unroll
-            for (int k = 0; k < V; ++k) rbar.v[k] = sum_r.v[k] / P.n_f;
+            for (int k = 0; k < V; ++k) rbar.v[k] = sum_r.v[k] / n_f;
             if constexpr (ERR) {
                 // Error reset (Algorithm 2 lines 11-12):
                 // x_i = (x_{i,t-1/2} - e_{i,t-1/2}) + mean_k e_{k,t-1/2}.
-                for (int i0 = 0; i0 < n; i0 += UF) {
-                    Pack<V> xv[UF];
+                for (int i0 = 0; i0 < n; i0 += UB) {
+                    Pack<V> xv[UB];
 #pragma unroll
-                    for (int u = 0; u < UF; ++u)
+                    for (int u = 0; u < UB; ++u)
                         if (i0 + u < n) xv[u] = ld<V>(x + (long long)(i0 + u) * d);
 #pragma unroll
-                    for (int u = 0; u < UF; ++u) {
+                    for (int u = 0; u < UB; ++u) {
                         if (i0 + u < n) {
 #pragma unroll
                             for (int k = 0; k < V; ++k) xv[u].v[k] = xv[u].v[k] + rbar.v[k];

@@ -99,8 +99,8 @@ def _run_both(d, n, bs, R1, R2, H, eta, beta, steps, seed=3, masks=None, x0=None
         opt.step(torch.from_numpy(g).to(DEV))
         ref.step(g)
         assert np.array_equal(opt.state(b.STATE_MASK_G).cpu().numpy(), ref.mask_g)
-        if t % H == 0:
-            assert np.array_equal(opt.state(b.STATE_MASK_R).cpu().numpy(), ref.mask_r)
+        if t >= H:      # the reset mask of the last reset step, also when read after later ordinary steps
+            assert np.array_equal(opt.state(b.STATE_MASK_R).cpu().numpy(), ref.mask_r), t
     return opt, ref
 
 
@@ -664,6 +664,92 @@ def test_random_shapes_parameters_and_flags_against_the_float32_oracle():
         opt.close()
 
 
+# ------------------------------------------------------------------ the opt-in staged selected-block kernel
+STAGED_SHAPES = [
+    # d, n, bs, R1, R2, H, beta, flags
+    (4096 + 40, 8, 256, 4, 4, 4, 0.0, 0),             # ragged last block
+    (4096 + 40, 8, 256, 4, 2, 3, 0.9, 0),
+    (20_000, 16, 1024, 2, 2, 2, 0.9, 0),              # n = 16: blocks cut into several chunks
+    (262_144 + 4, 8, 512, 32, 32, 8, 0.9, 0),         # the headline shape's geometry, tail of one vector column
+    (60_000, 8, 2048, 1, 1, 2, 0.9, 0),               # R = 1: dense walk, every block update- and reset-selected
+    (33_000, 3, 64, 2, 3, 1, 0.5, 0),                 # smallest staged block (16 vector columns), odd worker count
+    (50_000, 8, 512, 3, 2, 2, 0.9, 1),                # implementation II (no error array)
+    (50_000, 5, 512, 0, 2, 1, 0.0, 1),                # CSEA, implementation II, no momentum
+    (70_000, 24, 4096, 2, 2, 2, 0.9, 0),              # many workers: a stage holds 32 columns
+]
+
+
+@pytest.mark.parametrize("d,n,bs,R1,R2,H,beta,flags", STAGED_SHAPES)
+def test_staged_selected_block_kernel_equals_float32_oracle_exactly(d, n, bs, R1, R2, H, beta, flags):
+    """CSER_FLAG_STAGED_SELECTED: the shared-memory staged kernel must give the same bits as the oracle
+    (and hence as the default kernel) on update-selected, reset-selected and doubly selected blocks."""
+    impl2 = bool(flags & b.FLAG_NO_ERROR_ARRAY)
+    opt, ref = _run_both(d, n, bs, R1, R2, H, 0.1, beta, steps=9, flags=flags | b.FLAG_STAGED_SELECTED,
+                         oracle=CSERImpl2Oracle if impl2 else CSEROracle)
+    names = ((b.STATE_X, "x"),) + (() if impl2 else ((b.STATE_E, "e"),)) + (((b.STATE_M, "m"),) if beta else ())
+    for which, name in names:
+        got, want = opt.state(which).cpu().numpy(), getattr(ref, name)
+        assert np.array_equal(got, want), (name, int((got != want).sum()))
+    opt.close()
+
+
+def test_staged_kernel_with_injected_masks_replay_and_host_gradients():
+    """The staged kernel behind the other entry points: injected masks (all four combinations), replayable
+    steps (reset flag and list length read on the device) and host-gradient slabs (column ranges)."""
+    d, n, bs = 64 * 40 + 20, 4, 64
+    B = n_blocks(d, bs)
+    rng = np.random.default_rng(5)
+    masks = [(rng.integers(0, 2, B).astype(np.uint8), rng.integers(0, 2, B).astype(np.uint8)) for _ in range(4)]
+    opt, ref = _run_both(d, n, bs, 2, 2, 1, 0.1, 0.9, steps=4, masks=masks, flags=b.FLAG_STAGED_SELECTED)
+    for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e"), (b.STATE_M, "m")):
+        assert np.array_equal(opt.state(which).cpu().numpy(), getattr(ref, name)), name
+    opt.close()
+    w = synth.CONFIGS[2].scaled(d=1_200_000 + 4, steps=6)
+    a = b.CSER(w.d, w.n_workers, w.block_size, 4, 2, 3, w.eta, w.beta, 5, flags=b.FLAG_STAGED_SELECTED)
+    c = b.CSER(w.d, w.n_workers, w.block_size, 4, 2, 3, w.eta, w.beta, 5)
+    x0 = synth.x0(w, DEV)
+    a.set_x0(x0), c.set_x0(x0)
+    pinned = torch.empty((w.n_workers, w.d), dtype=torch.float32).pin_memory()
+    for t in range(1, w.steps + 1):
+        g = synth.gradients(w, t, DEV)
+        pinned.copy_(g)
+        if t == 3:
+            b.cser_replay_begin(a.h)
+            b.cser_step_replayable(a.h, g)
+            b.cser_replay_end(a.h)
+        elif t % 2:
+            a.step(g)
+        else:
+            a.step_host(pinned)
+        c.step(g)
+        torch.cuda.synchronize()
+    for which in (b.STATE_X, b.STATE_E, b.STATE_M):
+        assert torch.equal(a.state(which), c.state(which)), which
+    a.close(), c.close()
+
+
+# ------------------------------------------------------------------ C2 = 0 without an error array
+@pytest.mark.parametrize("H,R2,beta", [(1, 4, 0.0), (1, 2, 0.9), (4, 2, 0.9), (3, 1, 0.0)])
+def test_csea_and_cser_pl_in_implementation_II(H, R2, beta):
+    """R1 = 0 together with CSER_FLAG_NO_ERROR_ARRAY: the special cases of Appendix A.1 (CSEA for H = 1,
+    CSER-PL otherwise) in the form without an error array of Appendix A.4: nothing is exchanged between
+    resets and a reset replaces the reset-selected blocks of x by their mean over workers."""
+    d, n, bs = 4096 + 40, 8, 256
+    opt, ref = _run_both(d, n, bs, 0, R2, H, 0.1, beta, steps=9, flags=b.FLAG_NO_ERROR_ARRAY,
+                         oracle=CSERImpl2Oracle)
+    assert np.array_equal(opt.state(b.STATE_X).cpu().numpy(), ref.x)
+    if beta:
+        assert np.array_equal(opt.state(b.STATE_M).cpu().numpy(), ref.m)
+    # the models agree with implementation I's (same masks, same gradients) to rounding
+    one, ref1 = _run_both(d, n, bs, 0, R2, H, 0.1, beta, steps=9)
+    x2, x1 = opt.state(b.STATE_X).cpu().numpy().astype(np.float64), one.state(b.STATE_X).cpu().numpy().astype(np.float64)
+    assert np.abs(x2 - x1).max() <= 1e-4 * np.abs(x1).max()
+    if R2 == 1:     # delta_1 = 1: every reset makes all workers' models equal (local SGD with period H)
+        x = opt.state(b.STATE_X).cpu().numpy()
+        assert (x == x[0]).all()
+    opt.close(), one.close()
+
+
 # ------------------------------------------------------------------ boundary behaviour
 def test_host_gradient_entry_point_equals_device_entry_point():
     w = synth.CONFIGS[2].scaled(d=3_000_000 + 4, steps=10)
@@ -763,3 +849,28 @@ def test_errors_are_reported_not_raised_on_the_device():
     opt.step(torch.zeros((2, 100), device=DEV))
     assert opt.t == 1
     opt.close()
+
+
+def test_refused_steps_leave_the_counter_and_the_state_alone():
+    """A step that is refused (bad pointer, wrong kind of memory, misaligned) happens before the iteration
+    counter moves: interleaved with good steps it must leave t, the masks and the state exactly as on a
+    handle that never saw it."""
+    L = b.lib()
+    d, n, bs = 5000, 4, 64
+    a = b.CSER(d, n, bs, 4, 2, 2, 0.1, 0.9, 9)
+    c = b.CSER(d, n, bs, 4, 2, 2, 0.1, 0.9, 9)
+    x0 = torch.randn(d, device=DEV)
+    a.set_x0(x0), c.set_x0(x0)
+    host = torch.zeros((n, d))
+    odd = torch.zeros(n * d + 1, device=DEV)
+    for t in range(1, 7):
+        g = torch.randn((n, d), device=DEV)
+        assert L.cser_step(a.h, None, None) == -1
+        assert L.cser_step(a.h, ctypes.c_void_p(host.data_ptr()), None) == -1
+        assert L.cser_step(a.h, ctypes.c_void_p(odd.data_ptr() + 2), None) == -1
+        assert a.t == t - 1
+        a.step(g), c.step(g)
+        assert a.t == c.t == t
+    for which in (b.STATE_X, b.STATE_E, b.STATE_M, b.STATE_MASK_G, b.STATE_MASK_R):
+        assert torch.equal(a.state(which), c.state(which)), which
+    a.close(), c.close()

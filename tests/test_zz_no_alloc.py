@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import CSEROracle
 from paper_2007_13221_b200 import binding as b, synth
 
 pytestmark = pytest.mark.gpu
@@ -39,6 +40,58 @@ def test_noalloc_step_equals_handle_step_on_consecutive_calls(beta, d):
         assert torch.equal(ref.state(b.STATE_E), e), t
         if beta:
             assert torch.equal(ref.state(b.STATE_M), m), t
+    ref.close()
+
+
+def test_noalloc_step_equals_the_float32_oracle():
+    """Directly against the CPU oracle (float32 evaluation, same operation order: equal bits), not only
+    against the handle-based entry point."""
+    torch.cuda.set_device(0)
+    d, n, bs, R1, R2, H, eta, beta, seed = 30_000 + 12, 5, 128, 3, 2, 2, 0.1, 0.9, 21
+    rng = np.random.default_rng(7)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    ref = CSEROracle(d, n, bs, R1, R2, H, eta, beta, seed, dtype=np.float32)
+    ref.set_x0(x0)
+    x = torch.from_numpy(np.tile(x0, (n, 1))).to(DEV)
+    e, m = torch.zeros_like(x), torch.zeros_like(x)
+    for t in range(1, 8):
+        g = rng.standard_normal((n, d)).astype(np.float32)
+        ref.step(g)
+        b.cser_step_noalloc(d, n, bs, R1, R2, H, eta, beta, seed, t, torch.from_numpy(g).to(DEV), x, e, m)
+        torch.cuda.synchronize()
+        for got, want, name in ((x, ref.x, "x"), (e, ref.e, "e"), (m, ref.m, "m")):
+            assert np.array_equal(got.cpu().numpy(), want), (t, name)
+
+
+def test_noalloc_at_its_largest_vector_on_a_side_stream_allocates_nothing():
+    """Exactly CSER_NOALLOC_MAX_BLOCKS blocks, every block selected (R1 = 1), so the list fills the
+    scratch to its last entry, right below the three counters; three or more consecutive steps on a side
+    stream, so that every counter takes its turn; and the free device memory does not move."""
+    torch.cuda.set_device(0)
+    max_blocks, bs, n = 262144, 4, 1
+    d = max_blocks * bs
+    R1, R2, H, eta, beta, seed = 1, 2, 1, 0.1, 0.0, 3
+    ref = b.CSER(d, n, bs, R1, R2, H, eta, beta, seed)
+    x0 = torch.randn(d, device=DEV)
+    ref.set_x0(x0)
+    x = x0[None, :].clone()
+    e = torch.zeros_like(x)
+    grads = [torch.randn((n, d), device=DEV) for _ in range(5)]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        b.cser_step_noalloc(d, n, bs, R1, R2, H, eta, beta, seed, 1, grads[0], x, e, None)   # warm-up call
+        side.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        for t in range(2, 6):
+            b.cser_step_noalloc(d, n, bs, R1, R2, H, eta, beta, seed, t, grads[t - 1], x, e, None)
+        side.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
+    for t in range(1, 6):
+        ref.step(grads[t - 1])
+    torch.cuda.synchronize()
+    assert torch.equal(ref.state(b.STATE_X), x)
+    assert torch.equal(ref.state(b.STATE_E), e)
     ref.close()
 
 
