@@ -34,6 +34,7 @@ NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2_wrn40x8_n8_R32_H8": 1.7983e9 * 35_748_708 
 NO_ERROR_ARRAY = False   # --impl2: implementation II of Appendix A.4 (no e array)
 EXACT_COUNT = False      # --exact-count: every mask selects exactly round(B/R) blocks
 L2_RESIDENT = False      # ask the library to keep a small state in L2 (CSER_FLAG_L2_RESIDENT)
+THREE_KERNELS = False    # --three-kernels: never the single-launch kernel for small problems (CSER_FLAG_THREE_KERNELS)
 STAGED = False           # --staged: selected blocks through the shared-memory staged kernel (CSER_FLAG_STAGED_SELECTED)
 
 
@@ -258,7 +259,7 @@ def run_workload(w, K, W, dev, rank, world, ring_n=0, with_e2e=True, flush_l2=Fa
     opt = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
                  block_begin=0 if EXACT_COUNT else rank * w.n_blocks,
                  flags=(b.FLAG_NO_ERROR_ARRAY if NO_ERROR_ARRAY else 0) | (b.FLAG_EXACT_COUNT if EXACT_COUNT else 0)
-                 | (b.FLAG_L2_RESIDENT if L2_RESIDENT else 0) | (b.FLAG_STAGED_SELECTED if STAGED else 0))
+                 | (b.FLAG_L2_RESIDENT if L2_RESIDENT else 0) | (b.FLAG_STAGED_SELECTED if STAGED else 0) | (b.FLAG_THREE_KERNELS if THREE_KERNELS else 0))
     opt.set_x0(synth.x0(w, dev))
     g_bytes = w.n_workers * w.d * 4
     ring_n = ring_n or max(2, min(4, int(6e9 // g_bytes)))
@@ -431,6 +432,8 @@ def main():
     ap.add_argument("--R1", type=int, default=-1, help="override the update compressor's ratio")
     ap.add_argument("--R2", type=int, default=-1, help="override the reset compressor's ratio")
     ap.add_argument("--H", type=int, default=-1, help="override the reset interval")
+    ap.add_argument("--three-kernels", action="store_true",
+                    help="small problems through the three-kernel step instead of the single-launch kernel")
     ap.add_argument("--staged", action="store_true",
                     help="selected blocks through the shared-memory staged kernel instead of the register-walking one")
     ap.add_argument("--flush-l2", action="store_true", help="per-kernel figures with L2 flushed between launches")
@@ -438,10 +441,11 @@ def main():
     ap.add_argument("--oracle-seconds", type=float, default=10.0, help=argparse.SUPPRESS)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
-    global NO_ERROR_ARRAY, EXACT_COUNT, STAGED
+    global NO_ERROR_ARRAY, EXACT_COUNT, STAGED, THREE_KERNELS
     NO_ERROR_ARRAY = bool(args.impl2)
     EXACT_COUNT = bool(args.exact_count)
     STAGED = bool(args.staged)
+    THREE_KERNELS = bool(args.three_kernels)
 
     from paper_2007_13221_b200 import synth
     w = synth.CONFIGS[args.config]

@@ -108,6 +108,7 @@ FLAG_NO_ERROR_ARRAY = 1
 FLAG_EXACT_COUNT = 2
 FLAG_L2_RESIDENT = 4
 FLAG_STAGED_SELECTED = 8
+FLAG_THREE_KERNELS = 16
 
 
 def cser_create(d, n_workers, block_size, R1, R2, H, eta, beta, seed, block_begin=0, flags=0):

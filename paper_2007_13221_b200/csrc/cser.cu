@@ -112,6 +112,7 @@ struct cser_ctx {
     // Its bounded waits report through err_host, one word of mapped pinned host memory that the host
     // looks at on every call without synchronizing.
     bool staging = false;
+    bool fused_small = true;                         // small problems as one launch (off with CSER_FLAG_THREE_KERNELS)
     int sm_count = 0;
     unsigned *err_host = nullptr, *err_dev = nullptr;
     float *x0_stage = nullptr;                       // [d] staging for a host x0
@@ -223,6 +224,15 @@ int select_for_iteration(cser_ctx *h, bool is_reset, cudaStream_t s) {
     return CSER_OK;
 }
 
+// Iterations that move at most this many bytes go through the single-launch kernel: below it the
+// kernel boundaries, events and stream waits of the three-kernel step cost more than its better use
+// of DRAM gains (about 10 us against 8 % of the traffic time; the two designs were measured to break
+// even at 235 to 300 MB per step).
+constexpr long long kFusedMaxBytes = 1ll << 28;
+long long step_bytes_bound(const cser_ctx *h) {
+    return (long long)h->n * h->d * (12 + (h->m ? 8 : 0) + (h->e ? 8 : 0));
+}
+
 // Work-unit geometry of the staged selected-block kernel: C vector columns per unit so that all n
 // workers' segments of every array fit one stage, blocks cut into equal chunks, as many stages as fit
 // the CTA's shared-memory budget.
@@ -304,7 +314,9 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     const bool stream_any = h->walk_all || h->R1 != 1;
     const bool have_aux = use_aux && h->aux != nullptr && h->n_total == 0;
     const bool beside = have_aux && stream_any;                       // selected-block kernel beside the streaming one
-    const bool prefetch = have_aux && !h->replay && h->n_buf == 2;    // next iteration's select kernel on aux
+    // next iteration's select kernel on aux (not where the single-launch kernel will run that iteration)
+    const bool prefetch = have_aux && !h->replay && h->n_buf == 2 &&
+                          !(h->fused_small && h->vec4 && !h->exact && step_bytes_bound(h) <= kFusedMaxBytes);
     const bool fork = beside || prefetch;
     if (fork) {
         CU_TRY(cudaEventRecord(h->ev_fork, s));
@@ -438,6 +450,8 @@ int launch_step(cser_ctx *h, const float *grad, long long col0, long long col1, 
     P.tiles = 0, P.rctl = nullptr;
     P.list_cap = (unsigned)h->B;
     P.chunk_cols = P.n_chunks = P.stages = 0, P.err_word = nullptr;
+    P.mask_g_out = P.mask_r_out = nullptr, P.block_begin = h->block_begin;
+    P.k0 = P.k1 = P.t_lo = P.t_hi = 0, P.R1 = h->R1, P.R2 = h->R2;
     P.d = h->d, P.n = h->n;
     P.eta = h->eta, P.beta = h->beta, P.n_f = (float)h->n;
     const bool v4 = h->vec4 && ((uintptr_t)grad % 16 == 0) && (col0 % 4 == 0) &&
@@ -450,6 +464,55 @@ int launch_step(cser_ctx *h, const float *grad, long long col0, long long col1, 
     P.c_begin = col0, P.c_end = col1, P.bsv = (unsigned)h->bs;
     P.cols_total = h->d;
     return launch_step_v<1>(h, P, is_reset, s, use_aux);
+}
+
+bool fused_applies(const cser_ctx *h, const float *grad) {
+    return h->fused_small && h->vec4 && !h->exact && !h->masks_injected && !h->replay && h->n_total == 0 &&
+           (uintptr_t)grad % 16 == 0 && step_bytes_bound(h) <= kFusedMaxBytes;
+}
+
+// The whole iteration h->t in one launch (small problems): masks drawn inside the kernel and recorded
+// in the current buffer set.
+int launch_fused_small(cser_ctx *h, const float *grad, bool is_reset, cudaStream_t s) {
+    if (int rc = join_prefetch(h, s)) return rc;       // a select kernel of an earlier three-kernel step
+    StepParams P = {};
+    P.g = grad, P.x = h->x, P.e = h->e, P.m = h->m;
+    P.d = h->d, P.n = h->n, P.cols_total = h->d / 4, P.c_begin = 0, P.c_end = h->d / 4;
+    P.bsv = (unsigned)(h->bs / 4), P.list_cap = (unsigned)h->B;
+    P.eta = h->eta, P.beta = h->beta, P.n_f = (float)h->n;
+    P.block_begin = h->block_begin, P.R1 = h->R1, P.R2 = h->R2;
+    P.k0 = (uint32_t)(h->seed & 0xffffffffu), P.k1 = (uint32_t)(h->seed >> 32);
+    P.t_lo = (uint32_t)(h->t & 0xffffffffu), P.t_hi = (uint32_t)(h->t >> 32);
+    P.mask_g_out = h->sb[h->cur].mask_g;
+    P.mask_r_out = reset_mask_of(h, h->t);
+    const unsigned grid = (unsigned)((P.cols_total + kWalkThreads - 1) / kWalkThreads);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeAccessPolicyWindow;
+    attr[0].val.accessPolicyWindow.base_ptr = h->state_base;
+    attr[0].val.accessPolicyWindow.num_bytes = h->state_bytes;
+    attr[0].val.accessPolicyWindow.hitRatio = 1.0f;
+    attr[0].val.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
+    attr[0].val.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid), cfg.blockDim = dim3(kWalkThreads), cfg.dynamicSmemBytes = 0, cfg.stream = s;
+    cfg.attrs = attr, cfg.numAttrs = h->l2_persist ? 1 : 0;
+    const bool mom = h->m != nullptr, err = h->e != nullptr;
+    void (*kernel)(const StepParams);
+    if (mom) {
+        if (err) kernel = is_reset ? cser_fused_small_kernel<true, true, true> : cser_fused_small_kernel<true, false, true>;
+        else     kernel = is_reset ? cser_fused_small_kernel<true, true, false> : cser_fused_small_kernel<true, false, false>;
+    } else {
+        if (err) kernel = is_reset ? cser_fused_small_kernel<false, true, true> : cser_fused_small_kernel<false, false, true>;
+        else     kernel = is_reset ? cser_fused_small_kernel<false, true, false> : cser_fused_small_kernel<false, false, false>;
+    }
+    CU_TRY(cudaLaunchKernelEx(&cfg, kernel, P));
+    h->launches++;
+    // what activate_selection does for the three-kernel step
+    h->mask_g = h->sb[h->cur].mask_g, h->sel_list = h->sb[h->cur].list;
+    if (is_reset) h->mask_r = h->last_mask_r = reset_mask_of(h, h->t);
+    h->pre_valid = false;
+    h->walk_all = false;
+    return CSER_OK;
 }
 
 int check_handle(cser_ctx *h) {
@@ -523,7 +586,7 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
         return nullptr;
     }
     if (flags & ~(uint32_t)(CSER_FLAG_NO_ERROR_ARRAY | CSER_FLAG_EXACT_COUNT | CSER_FLAG_L2_RESIDENT |
-                            CSER_FLAG_STAGED_SELECTED)) {
+                            CSER_FLAG_STAGED_SELECTED | CSER_FLAG_THREE_KERNELS)) {
         fail(CSER_ERR_INVALID, "cser_create: unknown flags 0x%x", flags);
         return nullptr;
     }
@@ -599,6 +662,7 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
         }
         h->staging = er == cudaSuccess;
     }
+    h->fused_small = !(flags & (CSER_FLAG_THREE_KERNELS | CSER_FLAG_STAGED_SELECTED));
     h->exact = (flags & CSER_FLAG_EXACT_COUNT) != 0;
     if (er == cudaSuccess && h->exact) er = cudaMalloc(&h->exact_scratch, sizeof(ExactScratch));
     if (er == cudaSuccess && h->exact) er = cudaMemset(h->exact_scratch, 0, sizeof(ExactScratch));
@@ -698,10 +762,11 @@ int cser_step(cser_handle h, const float *grad, void *stream) {
     const uint64_t t_before = h->t;
     const bool is_reset = begin_iteration(h);
     int rc = CSER_OK;
+    const bool fused = fused_applies(h, grad);
     if (h->timing && cudaEventRecord(h->ev[0], s) != cudaSuccess) rc = fail(CSER_ERR_CUDA, "cser_step: event record failed");
-    if (!rc) rc = select_for_iteration(h, is_reset, s);
+    if (!rc && !fused) rc = select_for_iteration(h, is_reset, s);
     if (!rc && h->timing && cudaEventRecord(h->ev[1], s) != cudaSuccess) rc = fail(CSER_ERR_CUDA, "cser_step: event record failed");
-    if (!rc) rc = launch_step(h, grad, 0, h->d, is_reset, s, true);
+    if (!rc) rc = fused ? launch_fused_small(h, grad, is_reset, s) : launch_step(h, grad, 0, h->d, is_reset, s, true);
     if (rc) return abandon_iteration(h, t_before, rc);
     if (h->timing) {
         CU_TRY(cudaEventRecord(h->ev[2], s));

@@ -60,6 +60,10 @@ struct StepParams {
     unsigned n_chunks;       // work units per block
     unsigned stages;         // stages of the copy ring
     unsigned *err_word;      // host-visible word a wait that ran out raises (may be NULL)
+    // single-launch kernel for small problems only (it draws the masks itself):
+    uint8_t *mask_g_out, *mask_r_out;
+    long long block_begin;   // global id of block 0
+    uint32_t k0, k1, t_lo, t_hi, R1, R2;
     int n;
     float eta, beta, n_f;
 };
@@ -108,13 +112,197 @@ constexpr double kDenseWalkFraction = CSER_DENSE_WALK_FRACTION;   // expected se
 // (p-bar and, if the block is reset-selected too, e-bar), the second writes x (and e) once; the e it
 // reads again was read a moment ago by the same thread and comes from cache.
 // This kernel has its own register budget; the streaming kernel stays at 32 registers.
+//
+// walk_selected_column: one vector column c of a block selected by the update mask (sg), the reset
+// mask (sr) or both.
+template <int V, bool MOM, bool RESET, bool ERR>
+__device__ __forceinline__ void walk_selected_column(const StepParams &P, long long c, bool sg, bool sr) {
+    constexpr int UA = CSER_WALK_UA, UB = CSER_WALK_UB, UR = CSER_WALK_UR;
+    const long long d = P.d;
+    const int n = P.n;
+    const float eta = P.eta, beta = P.beta, n_f = P.n_f;
+    Pack<V> zero;
+#pragma unroll
+    for (int k = 0; k < V; ++k) zero.v[k] = 0.f;
+    const float *__restrict__ g = P.g + c * V;
+    float *__restrict__ x = P.x + c * V;
+    float *__restrict__ e = ERR ? P.e + c * V : nullptr;
+    float *__restrict__ m = MOM ? P.m + c * V : nullptr;
+    if (sg) {
+        // Update-selected block (Algorithm 3 with C(v) = v): r = 0, p' = mean_k p_k.  First pass:
+        // the mean of p, m updated; if the block is reset-selected too (with an error array) the
+        // mean of e as well, e being unchanged by this step's update.
+        Pack<V> sum_p = zero, sum_r = zero;
+        const bool with_e = RESET && ERR && sr;
+        for (int i0 = 0; i0 < n; i0 += UA) {
+            Pack<V> gv[UA], mv[UA], ev[UA];
+#pragma unroll
+            for (int u = 0; u < UA; ++u) {
+                if (i0 + u < n) {
+                    const long long o = (long long)(i0 + u) * d;
+                    gv[u] = ld_stream<V>(g + o);
+                    if constexpr (MOM) mv[u] = ld<V>(m + o);
+                    if constexpr (RESET && ERR) {
+                        if (with_e) ev[u] = ld<V>(e + o);
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UA; ++u) {
+                if (i0 + u < n) {
+                    const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], eta, beta);
+                    if constexpr (MOM) st<V>(m + (long long)(i0 + u) * d, mv[u]);
+#pragma unroll
+                    for (int k = 0; k < V; ++k) {
+                        sum_p.v[k] = (i0 + u == 0) ? p.v[k] : sum_p.v[k] + p.v[k];
+                        if constexpr (RESET && ERR) {
+                            if (with_e) sum_r.v[k] = (i0 + u == 0) ? ev[u].v[k] : sum_r.v[k] + ev[u].v[k];
+                        }
+                    }
+                }
+            }
+        }
+        Pack<V> pbar, rbar = zero;
+#pragma unroll
+        for (int k = 0; k < V; ++k) pbar.v[k] = sum_p.v[k] / n_f;
+        if constexpr (RESET && !ERR) {
+            if (sr) {
+                // implementation II (Appendix A.4): x_i = mean_k (x_k - p-bar); one more pass over x
+                for (int i0 = 0; i0 < n; i0 += UB) {
+                    Pack<V> xv[UB];
+#pragma unroll
+                    for (int u = 0; u < UB; ++u)
+                        if (i0 + u < n) xv[u] = ld<V>(x + (long long)(i0 + u) * d);
+#pragma unroll
+                    for (int u = 0; u < UB; ++u) {
+                        if (i0 + u < n) {
+#pragma unroll
+                            for (int k = 0; k < V; ++k) {
+                                const float xh = xv[u].v[k] - pbar.v[k];
+                                sum_r.v[k] = (i0 + u == 0) ? xh : sum_r.v[k] + xh;
+                            }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < V; ++k) rbar.v[k] = sum_r.v[k] / n_f;
+                for (int i = 0; i < n; ++i) st<V>(x + (long long)i * d, rbar);
+                return;
+            }
+        }
+        if constexpr (RESET && ERR) {
+#pragma unroll
+            for (int k = 0; k < V; ++k) rbar.v[k] = sum_r.v[k] / n_f;
+        }
+        // Second pass: x_i -= p-bar, e untouched; on a reset-selected block (Algorithm 2 lines
+        // 11-12) x_i = ((x_i - p-bar) - e_i) + e-bar and e_i = 0.
+        for (int i0 = 0; i0 < n; i0 += UB) {
+            Pack<V> xv[UB], ev[UB];
+#pragma unroll
+            for (int u = 0; u < UB; ++u) {
+                if (i0 + u < n) {
+                    const long long o = (long long)(i0 + u) * d;
+                    xv[u] = ld<V>(x + o);
+                    if constexpr (RESET && ERR) {
+                        if (with_e) ev[u] = ld<V>(e + o);
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UB; ++u) {
+                if (i0 + u < n) {
+                    const long long o = (long long)(i0 + u) * d;
+#pragma unroll
+                    for (int k = 0; k < V; ++k) xv[u].v[k] = xv[u].v[k] - pbar.v[k];
+                    if constexpr (RESET && ERR) {
+                        if (with_e) {
+#pragma unroll
+                            for (int k = 0; k < V; ++k) xv[u].v[k] = (xv[u].v[k] - ev[u].v[k]) + rbar.v[k];
+                            st<V>(e + o, zero);
+                        }
+                    }
+                    st<V>(x + o, xv[u]);
+                }
+            }
+        }
+    } else if constexpr (RESET) {
+        // Selected by the reset mask only: take the residual step (x_{t-1/2} = x - p,
+        // e_{t-1/2} = e - p).  With an error array store x_{t-1/2} - e_{t-1/2}, zero e and
+        // gather sum_k e_{k,t-1/2}; without one gather sum_k x_{k,t-1/2}.  (Forming the sum in
+        // a pass of its own and writing x once was measured and is slower here: it reads g, m
+        // and e twice, and these blocks are too few for the re-reads to stay in L1.)
+        Pack<V> sum_r = zero;
+        for (int i0 = 0; i0 < n; i0 += UR) {
+            Pack<V> gv[UR], mv[UR], xv[UR], ev[UR];
+#pragma unroll
+            for (int u = 0; u < UR; ++u) {
+                if (i0 + u < n) {
+                    const long long o = (long long)(i0 + u) * d;
+                    gv[u] = ld_stream<V>(g + o);
+                    if constexpr (MOM) mv[u] = ld<V>(m + o);
+                    xv[u] = ld<V>(x + o);
+                    if constexpr (ERR) ev[u] = ld<V>(e + o);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UR; ++u) {
+                if (i0 + u < n) {
+                    const long long o = (long long)(i0 + u) * d;
+                    const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], eta, beta);
+                    if constexpr (MOM) st<V>(m + o, mv[u]);
+                    if constexpr (ERR) {
+#pragma unroll
+                        for (int k = 0; k < V; ++k) {
+                            const float xh = xv[u].v[k] - p.v[k];
+                            const float eh = ev[u].v[k] - p.v[k];
+                            sum_r.v[k] = (i0 + u == 0) ? eh : sum_r.v[k] + eh;
+                            xv[u].v[k] = xh - eh;
+                        }
+                        st<V>(x + o, xv[u]);
+                        st<V>(e + o, zero);
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < V; ++k) {
+                            const float xh = xv[u].v[k] - p.v[k];
+                            sum_r.v[k] = (i0 + u == 0) ? xh : sum_r.v[k] + xh;
+                        }
+                    }
+                }
+            }
+        }
+        Pack<V> rbar;
+#pragma unroll
+        for (int k = 0; k < V; ++k) rbar.v[k] = sum_r.v[k] / n_f;
+        if constexpr (ERR) {
+            // Error reset (Algorithm 2 lines 11-12):
+            // x_i = (x_{i,t-1/2} - e_{i,t-1/2}) + mean_k e_{k,t-1/2}.
+            for (int i0 = 0; i0 < n; i0 += UB) {
+                Pack<V> xv[UB];
+#pragma unroll
+                for (int u = 0; u < UB; ++u)
+                    if (i0 + u < n) xv[u] = ld<V>(x + (long long)(i0 + u) * d);
+#pragma unroll
+                for (int u = 0; u < UB; ++u) {
+                    if (i0 + u < n) {
+#pragma unroll
+                        for (int k = 0; k < V; ++k) xv[u].v[k] = xv[u].v[k] + rbar.v[k];
+                        st<V>(x + (long long)(i0 + u) * d, xv[u]);
+                    }
+                }
+            }
+        } else {
+            // Implementation II (Appendix A.4): x_i = mean_k x_{k,t-1/2} for every worker.
+            for (int i = 0; i < n; ++i) st<V>(x + (long long)i * d, rbar);
+        }
+    }
+}
+
 // DENSE = false: threads are laid over the listed blocks (few blocks selected).  DENSE =
 // true: one thread per column of the whole range, returning at once if no mask selects its
 // block; used when a large share of the blocks is selected, where walking the columns in
 // their natural order is worth more than the idle threads cost.
 template <int V, bool MOM, bool RESET, bool ERR, bool DENSE>
 __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepParams P) {
-    constexpr int UA = CSER_WALK_UA, UB = CSER_WALK_UB, UR = CSER_WALK_UR;
     const uint8_t *__restrict__ mask_g = P.mask_g;
     const uint8_t *__restrict__ mask_r = P.mask_r;
     const uint32_t *__restrict__ list = P.list;
@@ -125,12 +313,6 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
     const bool reset_on = RESET && (P.rctl ? P.rctl->c[0].reset != 0 : true);
     const unsigned long long total =
         DENSE ? (unsigned long long)(P.c_end - P.c_begin) : (unsigned long long)n_listed * P.bsv;
-    const long long d = P.d;
-    const int n = P.n;
-    const float eta = P.eta, beta = P.beta, n_f = P.n_f;
-    Pack<V> zero;
-#pragma unroll
-    for (int k = 0; k < V; ++k) zero.v[k] = 0.f;
     for (unsigned long long f = (unsigned long long)blockIdx.x * kWalkThreads + threadIdx.x; f < total;
          f += (unsigned long long)gridDim.x * kWalkThreads) {
         long long c;
@@ -147,179 +329,69 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
         }
         const bool sg = mask_g[blk] != 0;
         const bool sr = reset_on ? (mask_r[blk] != 0) : false;
-        if constexpr (DENSE) {
-            if (!sg && !sr) continue;
-        }
-        const float *__restrict__ g = P.g + c * V;
-        float *__restrict__ x = P.x + c * V;
-        float *__restrict__ e = ERR ? P.e + c * V : nullptr;
-        float *__restrict__ m = MOM ? P.m + c * V : nullptr;
+        if (sg || sr) walk_selected_column<V, MOM, RESET, ERR>(P, c, sg, sr);
+    }
+}
 
-        if (sg) {
-            // Update-selected block (Algorithm 3 with C(v) = v): r = 0, p' = mean_k p_k.  First pass:
-            // the mean of p, m updated; if the block is reset-selected too (with an error array) the
-            // mean of e as well, e being unchanged by this step's update.
-            Pack<V> sum_p = zero, sum_r = zero;
-            const bool with_e = RESET && ERR && sr;
-            for (int i0 = 0; i0 < n; i0 += UA) {
-                Pack<V> gv[UA], mv[UA], ev[UA];
+// Small problems (a step of a few tens of microseconds) are bound by launches, not by bandwidth: three
+// kernels, two events and two stream waits cost as much as the traffic.  For them the whole iteration
+// is ONE launch: a thread owns one vector column, draws its block's GRBS mask bits itself (Definition
+// 2: Philox keyed on seed, t, block; every thread of a block redoes the same few hundred integer
+// operations, which is cheaper than a kernel boundary), the first thread of each block records them
+// for cser_read_state, and the column is then walked over the workers: selected blocks as in the
+// selected-block kernel, unselected ones elementwise (x_i -= p_i, e_i -= p_i).
+template <bool MOM, bool RESET, bool ERR>
+__global__ void __launch_bounds__(kWalkThreads) cser_fused_small_kernel(const StepParams P) {
+    constexpr int V = 4, U = 2;
+    const long long c = (long long)blockIdx.x * kWalkThreads + threadIdx.x;
+    if (c >= P.cols_total) return;
+    const unsigned blk = (uint32_t)c / P.bsv;
+    const uint32_t gb = (uint32_t)(P.block_begin + blk);
+    bool sg = false, sr = false;
+    if (P.R1 != 0)
+        sg = (unsigned long long)philox4x32_10_word0(P.k0, P.k1, gb, P.t_lo, P.t_hi, 0u) * P.R1 < (1ull << 32);
+    if constexpr (RESET)
+        sr = (unsigned long long)philox4x32_10_word0(P.k0, P.k1, gb, P.t_lo, P.t_hi, 1u) * P.R2 < (1ull << 32);
+    if (c == (long long)blk * P.bsv) {
+        P.mask_g_out[blk] = sg ? 1 : 0;
+        if constexpr (RESET) P.mask_r_out[blk] = sr ? 1 : 0;
+    }
+    if (sg || sr) {
+        walk_selected_column<V, MOM, RESET, ERR>(P, c, sg, sr);
+        return;
+    }
+    // C(p) = 0 on this block, so p' = r = p (Algorithm 3 lines 4-8): x_i -= p_i, e_i -= p_i
+    const long long d = P.d;
+    const int n = P.n;
+    const float *__restrict__ g = P.g + c * V;
+    float *__restrict__ x = P.x + c * V;
+    float *__restrict__ e = ERR ? P.e + c * V : nullptr;
+    float *__restrict__ m = MOM ? P.m + c * V : nullptr;
+    for (int i0 = 0; i0 < n; i0 += U) {
+        Pack<V> gv[U], mv[U], xv[U], ev[U];
 #pragma unroll
-                for (int u = 0; u < UA; ++u) {
-                    if (i0 + u < n) {
-                        const long long o = (long long)(i0 + u) * d;
-                        gv[u] = ld_stream<V>(g + o);
-                        if constexpr (MOM) mv[u] = ld<V>(m + o);
-                        if constexpr (RESET && ERR) {
-                            if (with_e) ev[u] = ld<V>(e + o);
-                        }
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < UA; ++u) {
-                    if (i0 + u < n) {
-                        const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], eta, beta);
-                        if constexpr (MOM) st<V>(m + (long long)(i0 + u) * d, mv[u]);
-#pragma unroll
-                        for (int k = 0; k < V; ++k) {
-                            sum_p.v[k] = (i0 + u == 0) ? p.v[k] : sum_p.v[k] + p.v[k];
-                            if constexpr (RESET && ERR) {
-                                if (with_e) sum_r.v[k] = (i0 + u == 0) ? ev[u].v[k] : sum_r.v[k] + ev[u].v[k];
-                            }
-                        }
-                    }
-                }
+        for (int u = 0; u < U; ++u) {
+            if (i0 + u < n) {
+                const long long o = (long long)(i0 + u) * d;
+                gv[u] = ld_stream<V>(g + o);
+                if constexpr (MOM) mv[u] = ld<V>(m + o);
+                xv[u] = ld<V>(x + o);
+                if constexpr (ERR) ev[u] = ld<V>(e + o);
             }
-            Pack<V> pbar, rbar = zero;
+        }
 #pragma unroll
-            for (int k = 0; k < V; ++k) pbar.v[k] = sum_p.v[k] / n_f;
-            if constexpr (RESET && !ERR) {
-                if (sr) {
-                    // implementation II (Appendix A.4): x_i = mean_k (x_k - p-bar); one more pass over x
-                    for (int i0 = 0; i0 < n; i0 += UB) {
-                        Pack<V> xv[UB];
+        for (int u = 0; u < U; ++u) {
+            if (i0 + u < n) {
+                const long long o = (long long)(i0 + u) * d;
+                const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], P.eta, P.beta);
 #pragma unroll
-                        for (int u = 0; u < UB; ++u)
-                            if (i0 + u < n) xv[u] = ld<V>(x + (long long)(i0 + u) * d);
-#pragma unroll
-                        for (int u = 0; u < UB; ++u) {
-                            if (i0 + u < n) {
-#pragma unroll
-                                for (int k = 0; k < V; ++k) {
-                                    const float xh = xv[u].v[k] - pbar.v[k];
-                                    sum_r.v[k] = (i0 + u == 0) ? xh : sum_r.v[k] + xh;
-                                }
-                            }
-                        }
-                    }
-#pragma unroll
-                    for (int k = 0; k < V; ++k) rbar.v[k] = sum_r.v[k] / n_f;
-                    for (int i = 0; i < n; ++i) st<V>(x + (long long)i * d, rbar);
-                    continue;
+                for (int k = 0; k < V; ++k) {
+                    xv[u].v[k] = xv[u].v[k] - p.v[k];
+                    if constexpr (ERR) ev[u].v[k] = ev[u].v[k] - p.v[k];
                 }
-            }
-            if constexpr (RESET && ERR) {
-#pragma unroll
-                for (int k = 0; k < V; ++k) rbar.v[k] = sum_r.v[k] / n_f;
-            }
-            // Second pass: x_i -= p-bar, e untouched; on a reset-selected block (Algorithm 2 lines
-            // 11-12) x_i = ((x_i - p-bar) - e_i) + e-bar and e_i = 0.
-            for (int i0 = 0; i0 < n; i0 += UB) {
-                Pack<V> xv[UB], ev[UB];
-#pragma unroll
-                for (int u = 0; u < UB; ++u) {
-                    if (i0 + u < n) {
-                        const long long o = (long long)(i0 + u) * d;
-                        xv[u] = ld<V>(x + o);
-                        if constexpr (RESET && ERR) {
-                            if (with_e) ev[u] = ld<V>(e + o);
-                        }
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < UB; ++u) {
-                    if (i0 + u < n) {
-                        const long long o = (long long)(i0 + u) * d;
-#pragma unroll
-                        for (int k = 0; k < V; ++k) xv[u].v[k] = xv[u].v[k] - pbar.v[k];
-                        if constexpr (RESET && ERR) {
-                            if (with_e) {
-#pragma unroll
-                                for (int k = 0; k < V; ++k) xv[u].v[k] = (xv[u].v[k] - ev[u].v[k]) + rbar.v[k];
-                                st<V>(e + o, zero);
-                            }
-                        }
-                        st<V>(x + o, xv[u]);
-                    }
-                }
-            }
-        } else if constexpr (RESET) {
-            // Selected by the reset mask only: take the residual step (x_{t-1/2} = x - p,
-            // e_{t-1/2} = e - p).  With an error array store x_{t-1/2} - e_{t-1/2}, zero e and
-            // gather sum_k e_{k,t-1/2}; without one gather sum_k x_{k,t-1/2}.  (Forming the sum in
-            // a pass of its own and writing x once was measured and is slower here: it reads g, m
-            // and e twice, and these blocks are too few for the re-reads to stay in L1.)
-            Pack<V> sum_r = zero;
-            for (int i0 = 0; i0 < n; i0 += UR) {
-                Pack<V> gv[UR], mv[UR], xv[UR], ev[UR];
-#pragma unroll
-                for (int u = 0; u < UR; ++u) {
-                    if (i0 + u < n) {
-                        const long long o = (long long)(i0 + u) * d;
-                        gv[u] = ld_stream<V>(g + o);
-                        if constexpr (MOM) mv[u] = ld<V>(m + o);
-                        xv[u] = ld<V>(x + o);
-                        if constexpr (ERR) ev[u] = ld<V>(e + o);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < UR; ++u) {
-                    if (i0 + u < n) {
-                        const long long o = (long long)(i0 + u) * d;
-                        const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], eta, beta);
-                        if constexpr (MOM) st<V>(m + o, mv[u]);
-                        if constexpr (ERR) {
-#pragma unroll
-                            for (int k = 0; k < V; ++k) {
-                                const float xh = xv[u].v[k] - p.v[k];
-                                const float eh = ev[u].v[k] - p.v[k];
-                                sum_r.v[k] = (i0 + u == 0) ? eh : sum_r.v[k] + eh;
-                                xv[u].v[k] = xh - eh;
-                            }
-                            st<V>(x + o, xv[u]);
-                            st<V>(e + o, zero);
-                        } else {
-#pragma unroll
-                            for (int k = 0; k < V; ++k) {
-                                const float xh = xv[u].v[k] - p.v[k];
-                                sum_r.v[k] = (i0 + u == 0) ? xh : sum_r.v[k] + xh;
-                            }
-                        }
-                    }
-                }
-            }
-            Pack<V> rbar;
-#pragma unroll
-            for (int k = 0; k < V; ++k) rbar.v[k] = sum_r.v[k] / n_f;
-            if constexpr (ERR) {
-                // Error reset (Algorithm 2 lines 11-12):
-                // x_i = (x_{i,t-1/2} - e_{i,t-1/2}) + mean_k e_{k,t-1/2}.
-                for (int i0 = 0; i0 < n; i0 += UB) {
-                    Pack<V> xv[UB];
-#pragma unroll
-                    for (int u = 0; u < UB; ++u)
-                        if (i0 + u < n) xv[u] = ld<V>(x + (long long)(i0 + u) * d);
-#pragma unroll
-                    for (int u = 0; u < UB; ++u) {
-                        if (i0 + u < n) {
-#pragma unroll
-                            for (int k = 0; k < V; ++k) xv[u].v[k] = xv[u].v[k] + rbar.v[k];
-                            st<V>(x + (long long)(i0 + u) * d, xv[u]);
-                        }
-                    }
-                }
-            } else {
-                // Implementation II (Appendix A.4): x_i = mean_k x_{k,t-1/2} for every worker.
-                for (int i = 0; i < n; ++i) st<V>(x + (long long)i * d, rbar);
+                if constexpr (MOM) st<V>(m + o, mv[u]);
+                st<V>(x + o, xv[u]);
+                if constexpr (ERR) st<V>(e + o, ev[u]);
             }
         }
     }

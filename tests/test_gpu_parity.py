@@ -29,6 +29,25 @@ def _built():
     torch.cuda.set_device(0)
 
 
+@pytest.fixture(params=["one_launch_when_small", "three_kernels"])
+def launch_path(request, monkeypatch):
+    """Small problems (at most 256 MB moved per step) are stepped by one kernel that draws the masks itself; larger ones,
+    and small ones created with CSER_FLAG_THREE_KERNELS, by the select / streaming / selected-block
+    kernels.  A test that takes this fixture runs once on each path (same expected results)."""
+    if request.param == "three_kernels":
+        create = b.cser_create
+
+        def create_three(*args, **kw):
+            args = list(args)
+            if len(args) >= 11:
+                args[10] |= b.FLAG_THREE_KERNELS
+            else:
+                kw["flags"] = kw.get("flags", 0) | b.FLAG_THREE_KERNELS
+            return create(*args, **kw)
+        monkeypatch.setattr(b, "cser_create", create_three)
+    return request.param
+
+
 def _within(got, want, rtol, atol):
     return np.abs(got.astype(np.float64) - want) <= rtol * np.abs(want) + atol
 
@@ -119,7 +138,7 @@ SHAPES = [
 
 
 @pytest.mark.parametrize("d,n,bs,R1,R2,H,beta", SHAPES)
-def test_small_shapes_equal_float32_oracle_exactly(d, n, bs, R1, R2, H, beta):
+def test_small_shapes_equal_float32_oracle_exactly(d, n, bs, R1, R2, H, beta, launch_path):
     opt, ref = _run_both(d, n, bs, R1, R2, H, 0.1, beta, steps=13)
     for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e")) + (((b.STATE_M, "m"),) if beta else ()):
         got = opt.state(which).cpu().numpy()
@@ -132,7 +151,7 @@ def test_small_shapes_equal_float32_oracle_exactly(d, n, bs, R1, R2, H, beta):
 
 
 @pytest.mark.parametrize("d,n,bs,R1,R2,H,beta", SHAPES[:4])
-def test_small_shapes_within_stated_tolerance_of_float64_oracle(d, n, bs, R1, R2, H, beta):
+def test_small_shapes_within_stated_tolerance_of_float64_oracle(d, n, bs, R1, R2, H, beta, launch_path):
     for steps, rtol, atol_rms in ((1, 1e-6, None), (100, 1e-4, 1e-4)):
         opt, ref = _run_both(d, n, bs, R1, R2, H, 0.1, beta, steps=steps, dtype=np.float64)
         for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e")) + (((b.STATE_M, "m"),) if beta else ()):
@@ -162,7 +181,7 @@ def test_hand_worked_example_on_gpu(beta):
     opt.close()
 
 
-def test_all_four_mask_combinations_on_one_reset_step():
+def test_all_four_mask_combinations_on_one_reset_step(launch_path):
     """Blocks in neither / update only / reset only / both masks, vector and scalar paths."""
     for d, bs in ((64, 16), (62, 15)):
         B = n_blocks(d, bs)
@@ -271,7 +290,7 @@ def _full_size_parity(cfg, steps=None, n_random=192, impl2=False):
     torch.cuda.empty_cache()
 
 
-def test_config1_full_vector_every_element():
+def test_config1_full_vector_every_element(launch_path):
     """d = 2^20, n = 8, 20 steps: the whole state against the oracle, not a sample."""
     w = synth.CONFIGS[1]
     opt = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed)
@@ -315,7 +334,7 @@ def test_config5_bert_large_sized_on_sampled_blocks():
 # ------------------------------------------------------------------ special cases and implementation II
 @pytest.mark.parametrize("d,n,bs,R2,H,beta", [(4096 + 40, 8, 256, 4, 1, 0.0), (4096 + 40, 8, 256, 2, 4, 0.9),
                                               (1001, 3, 7, 2, 2, 0.9), (20_000, 16, 1024, 1, 3, 0.0)])
-def test_no_update_sync_special_cases_csea_and_cser_pl(d, n, bs, R2, H, beta):
+def test_no_update_sync_special_cases_csea_and_cser_pl(d, n, bs, R2, H, beta, launch_path):
     """R1 = 0 (C2 = 0): CSEA when H = 1, CSER-PL otherwise (Appendix A.1)."""
     opt, ref = _run_both(d, n, bs, 0, R2, H, 0.1, beta, steps=13)
     for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e")) + (((b.STATE_M, "m"),) if beta else ()):
@@ -334,7 +353,7 @@ def test_no_update_sync_special_cases_csea_and_cser_pl(d, n, bs, R2, H, beta):
 
 
 @pytest.mark.parametrize("d,n,bs,R1,R2,H,beta", SHAPES)
-def test_implementation_II_equals_its_float32_oracle_exactly(d, n, bs, R1, R2, H, beta):
+def test_implementation_II_equals_its_float32_oracle_exactly(d, n, bs, R1, R2, H, beta, launch_path):
     opt, ref = _run_both(d, n, bs, R1, R2, H, 0.1, beta, steps=13, flags=b.FLAG_NO_ERROR_ARRAY,
                          oracle=CSERImpl2Oracle)
     for which, name in ((b.STATE_X, "x"),) + (((b.STATE_M, "m"),) if beta else ()):
@@ -346,7 +365,7 @@ def test_implementation_II_equals_its_float32_oracle_exactly(d, n, bs, R1, R2, H
     opt.close()
 
 
-def test_implementation_II_models_match_implementation_I():
+def test_implementation_II_models_match_implementation_I(launch_path):
     d, n, bs = 50_000 + 12, 8, 256
     a, ra = _run_both(d, n, bs, 4, 2, 4, 0.1, 0.9, steps=40)
     c, rc = _run_both(d, n, bs, 4, 2, 4, 0.1, 0.9, steps=40, flags=b.FLAG_NO_ERROR_ARRAY, oracle=CSERImpl2Oracle)
@@ -418,14 +437,14 @@ def test_exact_count_mode_equals_its_float32_oracle_exactly(d, n, bs, R1, R2, H,
     (40_000, 64, 128, 16, 8, 2, 0.9),  # many workers
     (1 << 16, 2, 1 << 16, 2, 2, 2, 0.9),   # a single huge block
 ])
-def test_edge_shapes_equal_float32_oracle_exactly(d, n, bs, R1, R2, H, beta):
+def test_edge_shapes_equal_float32_oracle_exactly(d, n, bs, R1, R2, H, beta, launch_path):
     opt, ref = _run_both(d, n, bs, R1, R2, H, 0.1, beta, steps=7)
     for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e")) + (((b.STATE_M, "m"),) if beta else ()):
         assert np.array_equal(opt.state(which).cpu().numpy(), getattr(ref, name)), name
     opt.close()
 
 
-def test_steps_on_a_side_stream_and_kernel_timing_hooks():
+def test_steps_on_a_side_stream_and_kernel_timing_hooks(launch_path):
     w = synth.CONFIGS[2].scaled(d=300_000, steps=6)
     side = torch.cuda.Stream()
     a = b.CSER(w.d, w.n_workers, w.block_size, 4, 2, 2, w.eta, w.beta, 8)
@@ -444,15 +463,18 @@ def test_steps_on_a_side_stream_and_kernel_timing_hooks():
             assert 0.0 <= sel_ms < 50.0 and 0.0 < step_ms < 50.0
     side.synchronize()
     torch.cuda.synchronize()
-    # per step: selected-block kernel, streaming kernel and the NEXT step's select kernel; the first
-    # step also runs its own select kernel
-    assert b.cser_launch_count(c.h) - n0 == 3 * len(grads) + 1
+    if launch_path == "three_kernels":
+        # per step: selected-block kernel, streaming kernel and the NEXT step's select kernel; the first
+        # step also runs its own select kernel
+        assert b.cser_launch_count(c.h) - n0 == 3 * len(grads) + 1
+    else:
+        assert b.cser_launch_count(c.h) - n0 == len(grads)      # small problem: one kernel per step
     for which in (b.STATE_X, b.STATE_E, b.STATE_M):
         assert torch.equal(a.state(which), c.state(which))
     a.close(), c.close()
 
 
-def test_learning_rate_schedule_and_column_reads():
+def test_learning_rate_schedule_and_column_reads(launch_path):
     d, n, bs = 10_000, 4, 64
     rng = np.random.default_rng(8)
     x0 = rng.standard_normal(d).astype(np.float32)
@@ -487,7 +509,7 @@ def test_learning_rate_schedule_and_column_reads():
     opt.close()
 
 
-def test_two_handles_stepping_concurrently_on_two_streams():
+def test_two_handles_stepping_concurrently_on_two_streams(launch_path):
     w = synth.CONFIGS[2].scaled(d=1_000_000, steps=12)
     seeds = (31, 32)
     ref = [b.CSER(w.d, w.n_workers, w.block_size, 8, 4, 3, w.eta, w.beta, s) for s in seeds]
@@ -512,7 +534,7 @@ def test_two_handles_stepping_concurrently_on_two_streams():
     [h.close() for h in ref + par]
 
 
-def test_l2_resident_state_gives_the_same_results():
+def test_l2_resident_state_gives_the_same_results(launch_path):
     w = synth.CONFIGS[1].scaled(d=300_000, steps=9)          # 9.6 MB of state: fits the L2 set-aside
     a = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, 3)
     c = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, 3, flags=b.FLAG_L2_RESIDENT)
@@ -636,6 +658,7 @@ def test_random_shapes_parameters_and_flags_against_the_float32_oracle():
         exact = rng.random() < 0.3
         seed = int(rng.integers(0, 2**62))
         flags = (b.FLAG_NO_ERROR_ARRAY if impl2 else 0) | (b.FLAG_EXACT_COUNT if exact else 0)
+        flags |= b.FLAG_THREE_KERNELS if rng.random() < 0.4 else 0
         opt = b.CSER(d, n, bs, R1, R2, H, eta, beta, seed, flags=flags)
         ref = (CSERImpl2Oracle if impl2 else CSEROracle)(d, n, bs, R1, R2, H, eta, beta, seed, dtype=np.float32,
                                                          exact_count=exact)
@@ -730,7 +753,7 @@ def test_staged_kernel_with_injected_masks_replay_and_host_gradients():
 
 # ------------------------------------------------------------------ C2 = 0 without an error array
 @pytest.mark.parametrize("H,R2,beta", [(1, 4, 0.0), (1, 2, 0.9), (4, 2, 0.9), (3, 1, 0.0)])
-def test_csea_and_cser_pl_in_implementation_II(H, R2, beta):
+def test_csea_and_cser_pl_in_implementation_II(H, R2, beta, launch_path):
     """R1 = 0 together with CSER_FLAG_NO_ERROR_ARRAY: the special cases of Appendix A.1 (CSEA for H = 1,
     CSER-PL otherwise) in the form without an error array of Appendix A.4: nothing is exchanged between
     resets and a reset replaces the reset-selected blocks of x by their mean over workers."""
@@ -751,7 +774,7 @@ def test_csea_and_cser_pl_in_implementation_II(H, R2, beta):
 
 
 # ------------------------------------------------------------------ boundary behaviour
-def test_host_gradient_entry_point_equals_device_entry_point():
+def test_host_gradient_entry_point_equals_device_entry_point(launch_path):
     w = synth.CONFIGS[2].scaled(d=3_000_000 + 4, steps=10)
     a = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, 5)
     c = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, 5)
@@ -769,7 +792,7 @@ def test_host_gradient_entry_point_equals_device_entry_point():
     a.close(), c.close()
 
 
-def test_column_slabs_reproduce_the_whole_vector():
+def test_column_slabs_reproduce_the_whole_vector(launch_path):
     """Two handles that each own a slab of whole blocks, with global block ids, and exchange nothing."""
     from paper_2007_13221_b200.shard import slab_of_rank
     w = synth.CONFIGS[3].scaled(d=100_000 + 8, steps=9)
@@ -795,7 +818,7 @@ def test_column_slabs_reproduce_the_whole_vector():
     [s.close() for _, _, s in slabs]
 
 
-def test_checkpoint_and_resume_is_bit_identical():
+def test_checkpoint_and_resume_is_bit_identical(launch_path):
     w = synth.CONFIGS[2].scaled(d=50_000, steps=30)
     a = b.CSER(w.d, w.n_workers, w.block_size, 4, 4, w.H, w.eta, w.beta, 2)
     a.set_x0(synth.x0(w, DEV))
@@ -851,7 +874,7 @@ def test_errors_are_reported_not_raised_on_the_device():
     opt.close()
 
 
-def test_refused_steps_leave_the_counter_and_the_state_alone():
+def test_refused_steps_leave_the_counter_and_the_state_alone(launch_path):
     """A step that is refused (bad pointer, wrong kind of memory, misaligned) happens before the iteration
     counter moves: interleaved with good steps it must leave t, the masks and the state exactly as on a
     handle that never saw it."""
