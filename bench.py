@@ -3,11 +3,15 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
 
-One "step" = one pass of the whole hot path (GRBS mask kernel + fused step kernel)
-over one [n, d] batch of synthetic gradients.  The headline workload is the
-WRN-40-8-sized configuration (d = 35,748,708, n = 8, R1 = R2 = 32, H = 8, beta = 0.9).
+One "step" = one pass of the whole hot path (GRBS block select + streaming kernel +
+selected-block kernel) over one [n, d] batch of synthetic gradients.  The headline
+workload is the largest single-GPU configuration, the BERT-large-sized one
+(d = 335,141,888, n = 8, R1 = R2 = 64, H = 8, beta = 0.9: 43 GB of g/x/e/m); the other
+four configurations are timed briefly in the same run and reported under "per_config".
 Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank owns one column slab
-of that size with global block ids and no data is exchanged ("weak" scaling).
+of that size with global block ids and no data is exchanged ("weak" scaling); the
+worker-sharded step (one all-reduce of the packed selected blocks per iteration) is
+timed beside it and reported under "worker_sharded".
 """
 import argparse
 import json
@@ -25,10 +29,11 @@ UNIT = "steps/s"
 PEAK_NOMINAL_GBS = 8000.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per step of the streaming kernel plus the selected-block
-# kernel.  Captured with ncu on the same workload cut to d = 8,388,608 (1.7658e9 + 0.0325e9 bytes per
-# step) and scaled by d, traffic being proportional to d; see
-# profiles/cser_stream_and_selected_kernels_cfg2_d8M_ncu_full.md.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2_wrn40x8_n8_R32_H8": 1.7983e9 * 35_748_708 / 8_388_608}
+# kernel, from ncu captures of the same workloads cut to d = 8,388,608 and scaled by d (every byte is
+# touched once, so traffic is proportional to d).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2_wrn40x8_n8_R32_H8": 1.7983e9 * 35_748_708 / 8_388_608,
+                                "cfg5_bertlarge_n8_R64_H8": 1.8013e9 * 335_141_888 / 8_388_608}
+HEADLINE_CONFIG = 5
 
 
 NO_ERROR_ARRAY = False   # --impl2: implementation II of Appendix A.4 (no e array)
@@ -121,40 +126,77 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(s)}
 
 
-def oracle_sample_rate(w, target_seconds=15.0, sample_cols=1 << 18):
-    """Time the CPU oracle, as it stands, on a contiguous slab of whole blocks of workload w.
-    Returns (full-vector steps/s equivalent, description, threads used)."""
-    import numpy as np
-    import torch
-    from oracle import CSEROracle
-    from paper_2007_13221_b200 import synth
-    cols_n = min(w.d, sample_cols // w.block_size * w.block_size)
-    ws = w.scaled(cols_n)
-    ref = CSEROracle(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
-                     dtype=np.float64, cols=np.arange(cols_n))
-    ref.set_x0(synth.x0(ws, "cpu").numpy())
-    grads = [synth.gradients(ws, t, "cpu").numpy() for t in range(1, 5)]
-    ref.step(grads[0])                                    # warm-up (page faults, imports)
-    n_steps, t0 = 0, time.perf_counter()
-    while True:
-        ref.step(grads[n_steps % len(grads)])
-        n_steps += 1
-        el = time.perf_counter() - t0
-        if el >= target_seconds or n_steps >= 400:
-            break
-    rate = n_steps / el * (cols_n / w.d)
-    desc = (f"{n_steps} oracle steps (float64 NumPy) on the first {cols_n} of {w.d} columns x {w.n_workers} "
-            f"workers of {w.name}; rate scaled by {cols_n}/{w.d} to the full vector")
-    return rate, desc, 1, el
+ORACLE_SAMPLE_ELEM_WORKERS = 1 << 25      # about 2.5 s of oracle time per step on one host core
+
+
+def oracle_sample_cols(w):
+    """Columns of the contiguous slab of whole blocks the oracle is timed on: the whole vector when it is
+    small (workload 1 runs real full-d steps), else 2^25 element-workers' worth of it: float64 [n, cols]
+    arrays of 268 MB each, far larger than the host's caches, and a few seconds of oracle time per step."""
+    if w.n_workers * w.d <= ORACLE_SAMPLE_ELEM_WORKERS:
+        return w.d
+    return max(w.block_size, ORACLE_SAMPLE_ELEM_WORKERS // w.n_workers // w.block_size * w.block_size)
+
+
+class OracleSample:
+    """The CPU oracle, as it stands, on the first `cols` columns of workload w (columns are independent
+    given the masks, and the masks are those of the whole vector)."""
+
+    def __init__(self, w, cols, n_grads=3):
+        import numpy as np
+        from oracle import CSEROracle
+        from paper_2007_13221_b200 import synth
+        self.w, self.cols = w, cols
+        ws = w.scaled(cols)
+        self.ref = CSEROracle(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
+                              dtype=np.float64, cols=np.arange(cols))
+        self.ref.set_x0(synth.x0(ws, "cpu").numpy())
+        self.grads = [synth.gradients(ws, t, "cpu").numpy() for t in range(1, n_grads + 1)]
+        self.k = 0
+
+    def step(self):
+        """One oracle step; returns its wall time in seconds."""
+        t0 = time.perf_counter()
+        self.ref.step(self.grads[self.k % len(self.grads)])
+        self.k += 1
+        return time.perf_counter() - t0
+
+
+def oracle_sample_rate(w, target_seconds=15.0):
+    """Time the oracle on a bounded sample of workload w.  Returns a dict: measured slab, wall time,
+    steps, and the rate scaled to the full vector (work is proportional to the columns)."""
+    cols = oracle_sample_cols(w)
+    smp = OracleSample(w, cols)
+    smp.step()                                            # warm-up (page faults, imports)
+    walls = []
+    while sum(walls) < target_seconds and len(walls) < 400:
+        walls.append(smp.step())
+    wall = sum(walls)
+    rate_slab = len(walls) / wall
+    return {"value": rate_slab * (cols / w.d), "unit": UNIT, "cores": 1, "kind": "oracle",
+            "extrapolated": cols != w.d, "measured_cols": cols, "measured_steps": len(walls),
+            "measured_wall_s": wall, "measured_steps_per_s_on_slab": rate_slab,
+            "sample": (f"{len(walls)} steps of the float64 NumPy oracle on the first {cols} of {w.d} columns x "
+                       f"{w.n_workers} workers of {w.name} ({8 * w.n_workers * cols / 1e6:.0f} MB per float64 array)"
+                       + ("" if cols == w.d else f"; rate scaled by {cols}/{w.d} to the full vector"))}
+
+
+ALL_CORES_SLAB_COLS = 1 << 20     # per process: 67 MB per float64 [8, cols] array, beyond any cache level
+
+
+def all_cores_slab_cols(w, cores):
+    cols = min(ALL_CORES_SLAB_COLS, max(w.block_size, w.d // cores))
+    return max(w.block_size, cols // w.block_size * w.block_size)
 
 
 def oracle_all_cores(w, seconds=10.0):
-    """The same oracle with the columns split over all host cores: one process per core, each
-    timing its own slab of whole blocks at the same moment.  Returns (steps/s, description, cores)."""
+    """The same oracle with the columns split over all host cores: one process per core, each timing its
+    own slab of whole blocks at the same moment.  Returns a dict like oracle_sample_rate's."""
     import subprocess
     cores = min(os.cpu_count() or 1, 32)       # one Python process per core; keep the memory bounded
     procs = [subprocess.Popen([sys.executable, os.path.abspath(__file__), "--config", str(w_index(w)),
-                               "--oracle-slab", str(k), "--oracle-seconds", str(seconds)] +
+                               "--oracle-slab", str(k), "--oracle-cores", str(cores),
+                               "--oracle-seconds", str(seconds)] +
                               (["--d", str(w.d)] if w.d != base_config(w).d else []),
                               stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True,
                               env={**os.environ, "OMP_NUM_THREADS": "1", "MKL_NUM_THREADS": "1",
@@ -168,9 +210,10 @@ def oracle_all_cores(w, seconds=10.0):
             ok += 1
         except Exception:
             pass
-    desc = (f"{ok} processes, one per core, each stepping the float64 NumPy oracle on its own 65,536-column slab "
-            f"of {w.name} for {seconds:.0f} s at the same time; rates (scaled to the full vector) added")
-    return total, desc, ok
+    cols = all_cores_slab_cols(w, cores)
+    return {"value": total, "unit": UNIT, "cores": ok, "extrapolated": True, "measured_cols": cols * ok,
+            "sample": (f"{ok} processes, one per core, each stepping the float64 NumPy oracle on its own {cols}-column "
+                       f"slab of {w.name} for {seconds:.0f} s at the same time; rates (scaled to the full vector) added")}
 
 
 def base_config(w):
@@ -186,13 +229,13 @@ def w_index(w):
     raise ValueError(w.name)
 
 
-def oracle_slab_worker(w, slab, seconds):
-    """Child of oracle_all_cores: times the oracle on columns [slab * 65536, (slab + 1) * 65536)."""
+def oracle_slab_worker(w, slab, cores, seconds):
+    """Child of oracle_all_cores: times the oracle on its own slab of whole blocks."""
     import numpy as np
     from oracle import CSEROracle
     from paper_2007_13221_b200 import synth
-    width = 65536 // w.block_size * w.block_size
-    c0 = (slab * width) % max(width, (w.d - width) // w.block_size * w.block_size)
+    width = all_cores_slab_cols(w, cores)
+    c0 = min(slab * width, max(0, (w.d - width) // w.block_size * w.block_size))
     cols = np.arange(c0, min(c0 + width, w.d))
     ws = w.scaled(cols.size)
     ref = CSEROracle(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
@@ -208,29 +251,48 @@ def oracle_slab_worker(w, slab, seconds):
     print(json.dumps({"rate": n_steps / el * (cols.size / w.d)}))
 
 
+def config_of(w, world):
+    """The `config` object of the JSON line: the same in both arms (it depends on the workload only)."""
+    per = 12 + (8 if w.beta != 0 else 0) + 8
+    return {"workload": w.name, "d": w.d, "n_workers": w.n_workers, "block_size": w.block_size,
+            "R1": w.R1, "R2": w.R2, "H": w.H, "eta": w.eta, "beta": w.beta,
+            "parallelism": f"column slabs x{world}, no collective",
+            "l2": f"inputs larger than L2: about {w.n_workers * w.d * per / 1e9:.2f} GB touched per step, "
+                  "gradient buffers cycled"}
+
+
 def run_reference(args, w):
-    """--impl reference: the oracle, timed on the host cores, same metric and workload."""
+    """--impl reference: the oracle, timed on the host cores, same metric and workload.  Each timed
+    step is one oracle step on a bounded slab (the whole vector for workload 1); `ms_per_step` is the
+    wall time of that measured step and `value` its rate scaled to the full vector."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    per_step_budget = 2.0
-    rates = []
+    cols = oracle_sample_cols(w)
+    smp = OracleSample(w, cols)
     t_all0 = time.perf_counter()
+    walls = []
     for k in range(args.warmup + args.steps):
-        rate, desc, cores, _ = oracle_sample_rate(w, target_seconds=per_step_budget, sample_cols=1 << 17)
+        dt = smp.step()
         if k >= args.warmup:
-            rates.append(rate)
-        if time.perf_counter() - t_all0 > 150:
+            walls.append(dt)
+        if time.perf_counter() - t_all0 > 170 and walls:
             break
-    value = len(rates) / sum(1.0 / r for r in rates)
+    wall = sum(walls)
+    rate_slab = len(walls) / wall
+    value = rate_slab * (cols / w.d)
+    sample = (f"each timed step = one step of the float64 NumPy oracle on the first {cols} of {w.d} columns x "
+              f"{w.n_workers} workers ({8 * w.n_workers * cols / 1e6:.0f} MB per float64 array)"
+              + ("" if cols == w.d else f"; value = measured rate x {cols}/{w.d}"))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / value, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "d": w.d, "n_workers": w.n_workers, "block_size": w.block_size,
-                   "R1": w.R1, "R2": w.R2, "H": w.H, "eta": w.eta, "beta": w.beta},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
-                         "sample": "each timed step = " + desc},
+        "steps": len(walls), "warmup": args.warmup, "ms_per_step": 1e3 * wall / len(walls),
+        "ms_per_step_is": "wall time of one measured oracle step on the slab" if cols != w.d else "wall time of one oracle step",
+        "extrapolated": cols != w.d, "measured_cols": cols, "measured_wall_s": wall,
+        "measured_steps_per_s_on_slab": rate_slab, "full_vector_ms_per_step_estimate": 1e3 / value,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": config_of(w, max(1, args.gpus)),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -351,24 +413,41 @@ def run_workload(w, K, W, dev, rank, world, ring_n=0, with_e2e=True, flush_l2=Fa
     return out
 
 
-def run_worker_sharded(w, K, W, dev):
-    """The worker-sharded step with this GPU holding all workers (message built, no peer to sum with)."""
+def run_worker_sharded(w, K, W, dev, group, world, rank):
+    """The worker-sharded step: this rank holds n / world of the workload's workers (all d columns), packs
+    the sum over them of the selected blocks, the message is all-reduced over the ranks (NCCL, through
+    torch.distributed; nothing to reduce when world == 1) and applied.  Timed on the device, max over ranks."""
     import torch
+    import torch.distributed as dist
     from paper_2007_13221_b200 import binding as b, synth
-    opt = b.WorkerShardedCSER(w.d, w.n_workers, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed)
+    from paper_2007_13221_b200.shard import workers_of_rank
+    first, n_local = workers_of_rank(w.n_workers, rank, world)
+    opt = b.WorkerShardedCSER(w.d, n_local, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
+                              group=group)
     opt.set_x0(synth.x0(w, dev))
-    ring = [synth.gradients(w, 1 + k, dev) for k in range(3)]
+    wl = w if world == 1 else __import__("dataclasses").replace(w, n_workers=n_local, seed=w.seed + 1000 * rank)
+    ring = [synth.gradients(wl, 1 + k, dev) for k in range(3)]
     for k in range(W):
         opt.step(ring[k % 3])
+    if world > 1:
+        dist.barrier(group=group)
     torch.cuda.synchronize()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
     for k in range(K):
         opt.step(ring[k % 3])
     ev1.record()
+    if world > 1:
+        dist.barrier(group=group)
     torch.cuda.synchronize()
     ms = ev0.elapsed_time(ev1) / K
-    out = {"steps_per_s": 1e3 / ms, "ms_per_step": ms, "steps": K,
+    if world > 1:
+        tt = torch.tensor([ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX, group=group)
+        ms = float(tt.item())
+    out = {"workload": w.name, "ranks": world, "workers_per_rank": n_local,
+           "steps_per_s": 1e3 / ms, "ms_per_step": ms, "steps": K, "scaling": "strong",
+           "collective": "none (one rank)" if world == 1 else "NCCL all-reduce (sum) of the packed message, fp32",
            "message_bytes_plain_step": 4 * b.cser_wshard_message_elems(opt.h, False),
            "message_bytes_reset_step": 4 * b.cser_wshard_message_elems(opt.h, True)}
     opt.close()
@@ -420,7 +499,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=8)
-    ap.add_argument("--config", type=int, default=2, help="workload 1..5 (2 = headline)")
+    ap.add_argument("--config", type=int, default=0,
+                    help="workload 1..5 (default: 5, the largest; 2 if the GPU has too little free memory)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -437,8 +517,11 @@ def main():
     ap.add_argument("--staged", action="store_true",
                     help="selected blocks through the shared-memory staged kernel instead of the register-walking one")
     ap.add_argument("--flush-l2", action="store_true", help="per-kernel figures with L2 flushed between launches")
+    ap.add_argument("--ceilings", action="store_true",
+                    help="measure the bandwidth ceilings and traversal / staging alternatives with the probe library")
     ap.add_argument("--oracle-slab", type=int, default=-1, help=argparse.SUPPRESS)
     ap.add_argument("--oracle-seconds", type=float, default=10.0, help=argparse.SUPPRESS)
+    ap.add_argument("--oracle-cores", type=int, default=1, help=argparse.SUPPRESS)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     global NO_ERROR_ARRAY, EXACT_COUNT, STAGED, THREE_KERNELS
@@ -448,6 +531,16 @@ def main():
     THREE_KERNELS = bool(args.three_kernels)
 
     from paper_2007_13221_b200 import synth
+    default_run = args.config == 0 and not args.d and args.R1 < 0 and args.R2 < 0 and args.H < 0
+    if args.config == 0:
+        args.config = HEADLINE_CONFIG
+        if args.impl == "ours":
+            import torch
+            need = synth.CONFIGS[HEADLINE_CONFIG].n_workers * synth.CONFIGS[HEADLINE_CONFIG].d * 4 * 5.3
+            if torch.cuda.is_available():
+                torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+                if torch.cuda.mem_get_info()[0] < need:
+                    args.config = 2
     w = synth.CONFIGS[args.config]
     if args.d:
         w = w.scaled(args.d)
@@ -457,10 +550,13 @@ def main():
                     H=args.H if args.H >= 0 else w.H)
         w = replace(w, name=f"{w.name}@R1={w.R1},R2={w.R2},H={w.H}")
     if args.oracle_slab >= 0:
-        oracle_slab_worker(w, args.oracle_slab, args.oracle_seconds)
+        oracle_slab_worker(w, args.oracle_slab, args.oracle_cores, args.oracle_seconds)
         return
     if args.impl == "reference":
         run_reference(args, w)
+        return
+    if args.ceilings:
+        run_ceilings(args)
         return
 
     import torch
@@ -482,109 +578,154 @@ def main():
         dist.barrier()
 
     K, W = args.steps, args.warmup
-    r = run_workload(w, K, W, dev, rank, world, ring_n=args.ring, with_e2e=not args.no_e2e,
+    big = w.n_workers * w.d * 4 > 8e9           # one [n, d] array above 8 GB: two gradient buffers, one host buffer
+    r = run_workload(w, K, W, dev, rank, world, ring_n=args.ring or (2 if big else 0), with_e2e=not args.no_e2e,
                      flush_l2=args.flush_l2)
     alg_bytes = r["alg_bytes"]
 
+    def brief(ro, steps):
+        """A few numbers per extra run, so that the whole line stays short."""
+        gbs = ro["alg_bytes"] / (ro["ms_per_step"] * 1e-3) / 1e9
+        rf = ro["roofline"]
+        out = {"steps_per_s": round(ro["value"], 2), "ms_per_step": round(ro["ms_per_step"], 5), "steps": steps,
+               "hbm_gbs_step": round(gbs, 1), "frac_of_8TBs": round(gbs / PEAK_NOMINAL_GBS, 4),
+               "roofline": {"bound": "hbm", "achieved": round(rf["achieved"], 1), "peak": rf["peak"], "unit": "GB/s",
+                            "frac": round(rf["frac"], 4), "l2_flushed": rf["l2_flushed_between_launches"],
+                            "traffic": rf["traffic"]},
+               "plain_ms": rf["plain_steps"] and round(rf["plain_steps"]["ms_mean"], 5),
+               "reset_ms": rf["reset_steps"] and round(rf["reset_steps"]["ms_mean"], 5),
+               "sm_mhz": ro["clocks"]["sm_mhz"]}
+        return out
+
     # the other workloads and variants, briefly (single GPU, default invocation only); a failure
     # here is recorded and never costs the headline line
-    others = None
-    if world == 1 and args.config == 2 and not args.d and not args.no_others and not args.impl2 \
-            and not args.exact_count and not args.staged and w is synth.CONFIGS[2]:
-        others = {}
+    per_config = None
+    if world == 1 and default_run and not args.no_others and not args.impl2 and not args.exact_count \
+            and not args.staged and not args.three_kernels:
+        per_config = {}
 
         def guarded(name, fn):
             try:
-                others[name] = fn()
+                per_config[name] = fn()
             except Exception as ex:  # noqa: BLE001
-                others[name] = "failed: " + repr(ex)[:200]
-                torch.cuda.empty_cache()
+                per_config[name] = "failed: " + repr(ex)[:200]
+            torch.cuda.empty_cache()
 
-        def variant(flag_name):
-            global NO_ERROR_ARRAY, EXACT_COUNT
+        def variant(wv, flag_name, steps=50):
+            global NO_ERROR_ARRAY, EXACT_COUNT, THREE_KERNELS, L2_RESIDENT
             try:
-                if flag_name == "impl2":
-                    NO_ERROR_ARRAY = True
-                else:
-                    EXACT_COUNT = True
-                ro = run_workload(w, 50, 5, dev, rank, world, with_e2e=False)
+                NO_ERROR_ARRAY, EXACT_COUNT = flag_name == "impl2", flag_name == "exact"
+                THREE_KERNELS, L2_RESIDENT = flag_name == "three_kernels", flag_name == "l2"
+                return brief(run_workload(wv, steps, 5, dev, rank, world, with_e2e=False,
+                                          flush_l2=wv is synth.CONFIGS[1]), steps)
             finally:
-                NO_ERROR_ARRAY = EXACT_COUNT = False
-            return {"steps_per_s": ro["value"], "ms_per_step": ro["ms_per_step"], "steps": 50,
-                    "hbm_gbs_step": ro["alg_bytes"] / (ro["ms_per_step"] * 1e-3) / 1e9,
-                    "hbm_frac_of_8TBs": ro["alg_bytes"] / (ro["ms_per_step"] * 1e-3) / 1e9 / PEAK_NOMINAL_GBS,
-                    "kernel_gbs": ro["roofline"]["achieved"], "kernel_frac_of_measured": ro["roofline"]["frac"]}
+                NO_ERROR_ARRAY = EXACT_COUNT = THREE_KERNELS = L2_RESIDENT = False
 
-        def other_workload(c):
-            wo = c if isinstance(c, synth.Workload) else synth.CONFIGS[c]
-            c = 0 if isinstance(c, synth.Workload) else c
+        def other_workload(wo):
             free, _ = torch.cuda.mem_get_info()
             if free < wo.n_workers * wo.d * 4 * 6.5:
                 return "skipped: not enough free device memory"
-            ko = 400 if c == 1 else (20 if c == 5 else 50)
-            ro = run_workload(wo, ko, 5, dev, rank, world, with_e2e=False, flush_l2=(c == 1))
-            return {
-                "steps_per_s": ro["value"], "ms_per_step": ro["ms_per_step"], "steps": ko,
-                "hbm_gbs_step": ro["alg_bytes"] / (ro["ms_per_step"] * 1e-3) / 1e9,
-                "hbm_frac_of_8TBs": ro["alg_bytes"] / (ro["ms_per_step"] * 1e-3) / 1e9 / PEAK_NOMINAL_GBS,
-                "kernel_gbs": ro["roofline"]["achieved"], "kernel_frac_of_measured": ro["roofline"]["frac"],
-                "kernel_l2_flushed": ro["roofline"]["l2_flushed_between_launches"],
-                "plain_steps": ro["roofline"]["plain_steps"], "reset_steps": ro["roofline"]["reset_steps"],
-                "clocks": ro["clocks"],
-                "note": ("state (67 MB) fits the 126 MB L2: steps/s is back to back over a 200 MB working set; "
-                         "the kernel figure is taken with L2 flushed between launches") if c == 1 else None}
+            ko = 400 if wo is synth.CONFIGS[1] else 50
+            # workload 1 (67 MB of state) fits the 126 MB L2: steps/s is back to back; the roofline figure
+            # is taken with L2 flushed between launches
+            return brief(run_workload(wo, ko, 5, dev, rank, world, with_e2e=False,
+                                      flush_l2=wo is synth.CONFIGS[1]), ko)
 
-        guarded(w.name + " worker-sharded entry points, one rank holding all workers",
-                lambda: run_worker_sharded(w, 50, 5, dev))
-        guarded(w.name + " exact-count GRBS", lambda: variant("exact"))
-        guarded(w.name + " implementation II (no error array, 20 B per element-worker)", lambda: variant("impl2"))
-        for c in (1, 3, 4, 5):
-            guarded(synth.CONFIGS[c].name, lambda c=c: other_workload(c))
+        w2 = synth.CONFIGS[2]
+        for c in (1, 2, 3, 4):
+            if synth.CONFIGS[c] is not w:
+                guarded(synth.CONFIGS[c].name, lambda c=c: other_workload(synth.CONFIGS[c]))
+        guarded(w2.name + " implementation II (no error array)", lambda: variant(w2, "impl2"))
+        guarded(w2.name + " exact-count GRBS", lambda: variant(w2, "exact"))
+        guarded(synth.CONFIGS[1].name + " three kernels instead of one launch",
+                lambda: variant(synth.CONFIGS[1], "three_kernels", 400))
+        guarded(w2.name + " worker-sharded entry points, one rank holding all workers",
+                lambda: run_worker_sharded(w2, 50, 5, dev, None, 1, 0))
+        for R in (1, 2, 4, 8):                      # small ratios: a large share of the blocks is selected
+            wr = replace_ratios(w2, R, R)
+            guarded(wr.name, lambda wr=wr: other_workload(wr))
         for rc, wt in synth.PAPER_TUNED.items():     # the paper's tuned (R_C2, R_C1, H) per overall ratio
             guarded(wt.name, lambda wt=wt: other_workload(wt))
+        guarded(w2.name + " step captured in a CUDA graph and replayed", lambda: run_graph_replay(w2, 100, dev))
 
-        def l2_resident():
-            global L2_RESIDENT
-            try:
-                L2_RESIDENT = True
-                return other_workload(1)
-            finally:
-                L2_RESIDENT = False
-        guarded(synth.CONFIGS[1].name + " with the state kept in L2 (CSER_FLAG_L2_RESIDENT)", l2_resident)
-        guarded(synth.CONFIGS[1].name + " step captured in a CUDA graph and replayed",
-                lambda: run_graph_replay(synth.CONFIGS[1], 2000, dev))
-        guarded(w.name + " step captured in a CUDA graph and replayed", lambda: run_graph_replay(w, 100, dev))
+    # worker-sharded deployment (the paper's own setting): the workload's n workers split over the ranks,
+    # one NCCL all-reduce of the packed selected blocks per step.  The column-slab number above stays the
+    # headline; this entry is there so that a multi-GPU run measures both shardings.
+    wshard = None
+    if world > 1 and not args.no_others:
+        try:
+            ws_w = synth.CONFIGS[2]
+            if ws_w.n_workers % world == 0:
+                wshard = run_worker_sharded(ws_w, min(K, 50), 5, dev, dist.group.WORLD, world, rank)
+            else:
+                wshard = f"skipped: {ws_w.n_workers} workers do not split evenly over {world} ranks"
+        except Exception as ex:  # noqa: BLE001
+            wshard = "failed: " + repr(ex)[:200]
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        rate, desc, cores, _ = oracle_sample_rate(w)
-        cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
-        rate_all, desc_all, cores_all = oracle_all_cores(w)
-        cpu["all_cores"] = {"value": rate_all, "unit": UNIT, "cores": cores_all, "sample": desc_all}
+        cpu = oracle_sample_rate(w)
+        cpu["all_cores"] = oracle_all_cores(w)
 
     if rank == 0:
+        cfg = config_of(w, world)
+        if args.impl2 or args.exact_count:
+            cfg["workload"] += (" implementation II" if args.impl2 else "") + (" exact-count GRBS" if args.exact_count else "")
         line = {
+            "per_config": per_config, "worker_sharded": wshard,
             "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name + (" implementation II" if args.impl2 else "")
-                       + (" exact-count GRBS" if args.exact_count else ""),
-                       "d": w.d, "n_workers": w.n_workers, "block_size": w.block_size,
-                       "R1": w.R1, "R2": w.R2, "H": w.H, "eta": w.eta, "beta": w.beta,
-                       "overall_compression_ratio": w.overall_ratio,
-                       "deployment_bytes_per_worker_step": w.comm_bytes_per_worker_step,
-                       "parallelism": f"column slabs x{world}, no collective",
-                       "l2": f"inputs larger than L2: {alg_bytes / 1e9:.2f} GB touched per step, "
-                             f"{r['ring_n']} gradient buffers cycled"},
+            "dtype": "f32", "data": "synthetic", "config": cfg,
+            "workload_notes": {"overall_compression_ratio": w.overall_ratio,
+                               "deployment_bytes_per_worker_step": w.comm_bytes_per_worker_step,
+                               "gradient_buffers_cycled": r["ring_n"]},
             "hbm_gbs_step": alg_bytes / (r["ms_per_step"] * 1e-3) / 1e9,
             "hbm_frac_of_8TBs": alg_bytes / (r["ms_per_step"] * 1e-3) / 1e9 / PEAK_NOMINAL_GBS,
             "algorithmic_bytes_per_step": alg_bytes,
             "roofline": r["roofline"], "cpu_baseline": cpu, "e2e": r["e2e"],
-            "gpu_launches": r["launches"], "clocks": r["clocks"], "other_workloads": others,
+            "gpu_launches": r["launches"], "clocks": r["clocks"],
         }
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_ceilings(args):
+    """--ceilings: what bounds the step kernels, re-measured with the probe library (plain kernels moving
+    the bytes of one M-CSER step over the WRN-40-8-sized arrays in different orders and through different
+    paths; see csrc/membw_probe.cu).  Prints one JSON object."""
+    import ctypes
+    import torch
+    import __graft_entry__
+    from paper_2007_13221_b200 import synth
+    __graft_entry__.build()
+    L = ctypes.CDLL(os.path.join(ROOT, "paper_2007_13221_b200", "libcser_probe.so"))
+    L.cser_probe_run.argtypes = [ctypes.c_int, ctypes.c_int] + [ctypes.c_void_p] * 4 + \
+        [ctypes.c_longlong, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_float), ctypes.c_void_p]
+    w = synth.CONFIGS[2] if not args.d else synth.CONFIGS[2].scaled(args.d)
+    n, d = w.n_workers, w.d
+    torch.cuda.set_device(0)
+    arrs = [torch.randn((n, d), device="cuda:0") * 0.01 for _ in range(4)]
+    elems = n * d
+    cases = [("read g, m, x, e (rows)", 0, 0, 16), ("write m, x, e (rows)", 1, 0, 12), ("copy g -> x (rows)", 2, 0, 8),
+             ("step mix 4 read + 3 written, row after row, plain 128-bit accesses", 3, 0, 28)]
+    cases += [(f"step mix, thread per column walking all workers, {u} workers in flight", 4, u, 28) for u in (1, 2, 4, 8)]
+    cases += [(f"step mix, row after row, bulk copies into shared memory, {kb} KB tiles", 5, kb, 28) for kb in (2, 4, 8)]
+    out = {"workload_shape": f"{n} x {d} fp32 per array ({elems * 4 / 1e9:.2f} GB)", "reps": args.steps, "patterns": []}
+    with ClockSampler(0) as clocks:
+        for name, pattern, variant, bytes_per in cases:
+            ms = ctypes.c_float()
+            rc = L.cser_probe_run(pattern, variant, *[a.data_ptr() for a in arrs], d, n, args.steps, ctypes.byref(ms), None)
+            out["patterns"].append({"pattern": name, "ms": round(ms.value, 4) if rc == 0 else None,
+                                    "GB_per_s": round(elems * bytes_per / (ms.value * 1e-3) / 1e9, 1) if rc == 0 else None,
+                                    "rc": rc})
+    out["clocks"] = clocks.summary()
+    print(json.dumps(out))
+
+
+def replace_ratios(w, R1, R2):
+    from dataclasses import replace
+    return replace(w, R1=R1, R2=R2, name=f"{w.name}@R1={R1},R2={R2}")
 
 
 if __name__ == "__main__":

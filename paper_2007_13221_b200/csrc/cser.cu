@@ -56,6 +56,7 @@ int fail(int code, const char *fmt, ...) {
 // ------------------------------------------------------------------ handle
 struct cser_ctx {
     long long d = 0, B = 0, block_begin = 0;
+    long long Bpad = 0;                              // B rounded up to 16: distance between the two buffer sets
     int n = 0, bs = 0, H = 0, device = 0;
     uint32_t R1 = 1, R2 = 1;
     float eta = 0.f, beta = 0.f;
@@ -93,7 +94,9 @@ struct cser_ctx {
     bool replay = false;
     // worker-sharded mode (cser_create_wshard): n = local workers, n_total = all ranks' workers
     int n_total = 0;
+    // ordered lists of the selected blocks, one set per mask buffer set (allocations of 2 B entries)
     uint32_t *pos_g = nullptr, *pos_r = nullptr, *olist_g = nullptr, *olist_r = nullptr;
+    bool lists_ready[2] = {false, false};            // set k holds the lists of the masks in buffer set k
     bool wshard_open = false;                        // pack done, apply pending
     bool wshard_reset = false;
     // exact-count GRBS (CSER_FLAG_EXACT_COUNT)
@@ -414,7 +417,7 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
         // the following iteration's masks and list, behind the selected-block kernel
         const unsigned sgrid = (unsigned)((h->B + 255) / 256);
         grbs_select_replay_kernel<<<sgrid, 256, 0, ws>>>(h->ctl, h->sb[0].mask_g, h->sb[0].mask_r, h->sb[0].list,
-                                                         h->B, h->B, h->block_begin,
+                                                         h->Bpad, h->B, h->block_begin,
                                                          (uint32_t)(h->seed & 0xffffffffu), (uint32_t)(h->seed >> 32),
                                                          h->R1, h->R2, (uint32_t)h->H);
         h->launches++;
@@ -627,14 +630,16 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
         if (beta != 0.f) h->m = reinterpret_cast<float *>(p);
     }
     // the two buffer sets lie B entries apart in one allocation per kind
-    if (er == cudaSuccess) er = cudaMalloc(&h->sb[0].mask_g, 2 * (size_t)B);
-    if (er == cudaSuccess) er = cudaMalloc(&h->sb[0].mask_r, 2 * (size_t)B);
-    if (er == cudaSuccess) er = cudaMalloc(&h->sb[0].list, 2 * (size_t)B * sizeof(uint32_t));
-    if (er == cudaSuccess) er = cudaMemset(h->sb[0].mask_g, 0, 2 * (size_t)B);
-    if (er == cudaSuccess) er = cudaMemset(h->sb[0].mask_r, 0, 2 * (size_t)B);
+    const size_t Bpad = ((size_t)B + 15) / 16 * 16;
+    h->Bpad = (long long)Bpad;
+    if (er == cudaSuccess) er = cudaMalloc(&h->sb[0].mask_g, 2 * Bpad);
+    if (er == cudaSuccess) er = cudaMalloc(&h->sb[0].mask_r, 2 * Bpad);
+    if (er == cudaSuccess) er = cudaMalloc(&h->sb[0].list, 2 * Bpad * sizeof(uint32_t));
+    if (er == cudaSuccess) er = cudaMemset(h->sb[0].mask_g, 0, 2 * Bpad);
+    if (er == cudaSuccess) er = cudaMemset(h->sb[0].mask_r, 0, 2 * Bpad);
     if (er == cudaSuccess) {
-        h->sb[1].mask_g = h->sb[0].mask_g + B, h->sb[1].mask_r = h->sb[0].mask_r + B;
-        h->sb[1].list = h->sb[0].list + B;
+        h->sb[1].mask_g = h->sb[0].mask_g + Bpad, h->sb[1].mask_r = h->sb[0].mask_r + Bpad;
+        h->sb[1].list = h->sb[0].list + Bpad;
         h->mask_r_half[0] = h->sb[0].mask_r, h->mask_r_half[1] = h->sb[1].mask_r;
     }
     if (er == cudaSuccess) er = cudaMemset(h->state_base, 0, h->state_bytes);
@@ -947,10 +952,10 @@ cser_handle cser_create_wshard(int64_t d, int32_t n_local, int32_t n_total, int3
     cser_ctx *h = cser_create_ex(d, n_local, block_size, R1, R2, H, eta, beta, seed, 0, CSER_FLAG_EXACT_COUNT);
     if (!h) return nullptr;
     h->n_total = n_total;
-    cudaError_t er = cudaMalloc(&h->pos_g, (size_t)h->B * sizeof(uint32_t));
-    if (er == cudaSuccess) er = cudaMalloc(&h->pos_r, (size_t)h->B * sizeof(uint32_t));
-    if (er == cudaSuccess) er = cudaMalloc(&h->olist_g, (size_t)h->B * sizeof(uint32_t));
-    if (er == cudaSuccess) er = cudaMalloc(&h->olist_r, (size_t)h->B * sizeof(uint32_t));
+    cudaError_t er = cudaMalloc(&h->pos_g, 2 * (size_t)h->B * sizeof(uint32_t));
+    if (er == cudaSuccess) er = cudaMalloc(&h->pos_r, 2 * (size_t)h->B * sizeof(uint32_t));
+    if (er == cudaSuccess) er = cudaMalloc(&h->olist_g, 2 * (size_t)h->B * sizeof(uint32_t));
+    if (er == cudaSuccess) er = cudaMalloc(&h->olist_r, 2 * (size_t)h->B * sizeof(uint32_t));
     if (er != cudaSuccess) {
         fail(er == cudaErrorMemoryAllocation ? CSER_ERR_NOMEM : CSER_ERR_CUDA, "cser_create_wshard: %s",
              cudaGetErrorString(er));
@@ -993,10 +998,23 @@ int launch_wshard(cser_ctx *h, ShardParams P, bool is_reset, bool pack, cudaStre
     return CSER_OK;
 }
 
+// Ordered lists of the masks in buffer set `buf` (those of iteration t), on stream s.
+int launch_ordered_lists(cser_ctx *h, int buf, bool is_reset, uint64_t t, cudaStream_t s) {
+    const size_t set = (size_t)buf * (size_t)h->B;
+    const unsigned grid = (unsigned)((h->B + kScanThreads - 1) / kScanThreads);
+    ordered_lists_kernel<<<grid, kScanThreads, 0, s>>>(h->sb[buf].mask_g, is_reset ? reset_mask_of(h, t) : nullptr, h->B,
+                                                       h->pos_g + set, h->pos_r + set, h->olist_g + set,
+                                                       h->olist_r + set);
+    h->launches++;
+    CU_TRY(cudaGetLastError());
+    return CSER_OK;
+}
+
 int wshard_params(cser_ctx *h, const float *grad, float *msg, bool *v4, ShardParams *P) {
     P->g = grad, P->x = h->x, P->e = h->e, P->m = h->m, P->msg = msg;
     P->mask_g = h->mask_g, P->mask_r = h->mask_r;
-    P->pos_g = h->pos_g, P->olist_g = h->olist_g, P->olist_r = h->olist_r;
+    const size_t set = (size_t)h->cur * (size_t)h->B;          // the lists of the current mask buffer set
+    P->pos_g = h->pos_g + set, P->olist_g = h->olist_g + set, P->olist_r = h->olist_r + set;
     P->d = h->d, P->n = h->n;
     P->k_g = exact_k(h->B, h->R1), P->k_r = exact_k(h->B, h->R2);
     P->eta = h->eta, P->beta = h->beta, P->n_total_f = (float)h->n_total;
@@ -1023,17 +1041,43 @@ int cser_wshard_pack(cser_handle h, const float *grad, float *msg, size_t msg_el
     cudaStream_t s = (cudaStream_t)stream;
     const uint64_t t_before = h->t;
     const bool is_reset = begin_iteration(h);
+    const bool prefetched = h->pre_valid && h->pre_t == h->t && !h->masks_injected;
     if (int rc = select_for_iteration(h, is_reset, s)) return abandon_iteration(h, t_before, rc);
-    ordered_lists_kernel<<<1, 1024, 0, s>>>(h->mask_g, h->mask_r, h->B, is_reset ? 1 : 0, h->pos_g, h->pos_r,
-                                            h->olist_g, h->olist_r);
-    h->launches++;
-    CU_TRY(cudaGetLastError());
-    if (int rc = launch_step(h, grad, 0, h->d, is_reset, s, false)) return rc;   // unselected blocks
+    if (!(prefetched && h->lists_ready[h->cur])) {
+        if (int rc = launch_ordered_lists(h, h->cur, is_reset, h->t, s)) return abandon_iteration(h, t_before, rc);
+    }
+    h->lists_ready[h->cur] = false;          // consumed by this step
+    // the pack kernel (selected blocks) beside the streaming kernel (unselected blocks): disjoint columns
+    const bool beside = h->aux != nullptr;
+    cudaStream_t ps = s;
+    if (beside) {
+        CU_TRY(cudaEventRecord(h->ev_fork, s));
+        CU_TRY(cudaStreamWaitEvent(h->aux, h->ev_fork, 0));
+        ps = h->aux;
+    }
     ShardParams P;
     bool v4;
     wshard_params(h, grad, msg, &v4, &P);
-    const int rc = v4 ? launch_wshard<4>(h, P, is_reset, true, s) : launch_wshard<1>(h, P, is_reset, true, s);
-    if (rc) return rc;
+    int rc = v4 ? launch_wshard<4>(h, P, is_reset, true, ps) : launch_wshard<1>(h, P, is_reset, true, ps);
+    if (!rc) rc = launch_step(h, grad, 0, h->d, is_reset, s, false);   // unselected blocks
+    if (beside) {
+        CU_TRY(cudaEventRecord(h->ev_join, h->aux));
+        CU_TRY(cudaStreamWaitEvent(s, h->ev_join, 0));
+    }
+    if (rc) return abandon_iteration(h, t_before, rc);
+    if (beside && h->n_buf == 2) {
+        // the next iteration's masks and ordered lists, on the auxiliary stream behind the join
+        const uint64_t t_next = h->t + 1;
+        const bool next_reset = (t_next % (uint64_t)h->H) == 0;
+        const int nb = h->cur ^ 1;
+        int prc = launch_select(h, nb, t_next, next_reset, true, h->aux, &h->pre_count);
+        if (!prc) prc = launch_ordered_lists(h, nb, next_reset, t_next, h->aux);
+        h->pre_valid = prc == CSER_OK;
+        h->lists_ready[nb] = prc == CSER_OK;
+        h->pre_t = t_next;
+        CU_TRY(cudaEventRecord(h->ev_pre, h->aux));
+        h->pre_pending = true;
+    }
     h->wshard_open = true;
     h->wshard_reset = is_reset;
     return CSER_OK;
@@ -1074,7 +1118,7 @@ int cser_replay_begin(cser_handle h, void *stream) {
     CU_TRY(cudaStreamSynchronize(s));   // c is on this function's stack
     // masks and list of iteration t + 1 into buffer set 1, published in block 1
     const unsigned grid = (unsigned)((h->B + 255) / 256);
-    grbs_select_replay_kernel<<<grid, 256, 0, s>>>(h->ctl, h->sb[0].mask_g, h->sb[0].mask_r, h->sb[0].list, h->B,
+    grbs_select_replay_kernel<<<grid, 256, 0, s>>>(h->ctl, h->sb[0].mask_g, h->sb[0].mask_r, h->sb[0].list, h->Bpad,
                                                    h->B, h->block_begin, (uint32_t)(h->seed & 0xffffffffu),
                                                    (uint32_t)(h->seed >> 32), h->R1, h->R2, (uint32_t)h->H);
     h->launches++;
@@ -1094,7 +1138,7 @@ int cser_step_replayable(cser_handle h, const float *grad, void *stream) {
     cudaStream_t s = (cudaStream_t)stream;
     // the iteration prepared during the last step becomes the current one
     replay_advance_kernel<<<(unsigned)((h->B + 255) / 256), 256, 0, s>>>(h->ctl, h->sb[0].mask_g, h->sb[0].mask_r,
-                                                                         h->sb[0].list, h->B, h->B);
+                                                                         h->sb[0].list, h->Bpad, h->B);
     h->launches++;
     CU_TRY(cudaGetLastError());
     return launch_step(h, grad, 0, h->d, true, s, true);

@@ -11,30 +11,54 @@
 // and each rank applies sum / n_total.  The message holds the update-selected blocks in
 // ascending block order and, on a reset step, the reset-selected blocks after them.
 
-// Exclusive scan of the two masks in block order (one CTA): pos_*[b] = selected blocks below b,
-// olist_* = the selected blocks in ascending order.
-__global__ void __launch_bounds__(1024)
-ordered_lists_kernel(const uint8_t *__restrict__ mask_g, const uint8_t *__restrict__ mask_r, long long B,
-                     int is_reset, uint32_t *__restrict__ pos_g, uint32_t *__restrict__ pos_r,
-                     uint32_t *__restrict__ olist_g, uint32_t *__restrict__ olist_r) {
-    __shared__ uint32_t part[2][1024];
-    const long long chunk = (B + blockDim.x - 1) / blockDim.x;
-    const long long b0 = min(B, (long long)threadIdx.x * chunk), b1 = min(B, b0 + chunk);
-    uint32_t cg = 0, cr = 0;
-    for (long long b = b0; b < b1; ++b) {
-        cg += mask_g[b] != 0;
-        if (is_reset) cr += mask_r[b] != 0;
-    }
-    part[0][threadIdx.x] = cg, part[1][threadIdx.x] = cr;
+// Exclusive scan of the two masks in block order: pos_*[b] = selected blocks below b, olist_* = the
+// selected blocks in ascending order.  One CTA per 1024 blocks; a CTA first counts the flags in front of
+// its own blocks (B bytes at most, from L2, four flags per load), then scans its own 1024.  No CTA waits
+// for another.  mask_r may be NULL (not a reset step).
+constexpr int kScanThreads = 1024;
+__device__ __forceinline__ uint32_t block_sum_1024(uint32_t v, uint32_t *warp_sums) {
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();                       // warp_sums may still be read from the previous use
+    if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = v;
     __syncthreads();
-    uint32_t og = 0, orr = 0;
-    for (int j = 0; j < (int)threadIdx.x; ++j) og += part[0][j], orr += part[1][j];
-    for (long long b = b0; b < b1; ++b) {
-        pos_g[b] = og;
-        if (mask_g[b]) olist_g[og++] = (uint32_t)b;
-        if (is_reset) {
-            pos_r[b] = orr;
-            if (mask_r[b]) olist_r[orr++] = (uint32_t)b;
+    uint32_t t = 0;
+    for (int w = 0; w < kScanThreads / 32; ++w) t += warp_sums[w];
+    return t;
+}
+
+__global__ void __launch_bounds__(kScanThreads)
+ordered_lists_kernel(const uint8_t *__restrict__ mask_g, const uint8_t *__restrict__ mask_r, long long B,
+                     uint32_t *__restrict__ pos_g, uint32_t *__restrict__ pos_r,
+                     uint32_t *__restrict__ olist_g, uint32_t *__restrict__ olist_r) {
+    __shared__ uint32_t warp_sums[kScanThreads / 32];
+    const long long first = (long long)blockIdx.x * kScanThreads;     // a multiple of 4: word loads stay aligned
+    const long long b = first + threadIdx.x;
+    for (int which = 0; which < 2; ++which) {
+        const uint8_t *__restrict__ mask = which ? mask_r : mask_g;
+        if (!mask) continue;
+        uint32_t *__restrict__ pos = which ? pos_r : pos_g;
+        uint32_t *__restrict__ olist = which ? olist_r : olist_g;
+        // flags in front of this CTA's blocks (flags are 0 / 1 bytes: dp4a adds four at a time)
+        const uint32_t *words = reinterpret_cast<const uint32_t *>(mask);
+        uint32_t part = 0;
+        for (long long w = threadIdx.x; w < first / 4; w += kScanThreads) part = __dp4a(words[w], 0x01010101u, part);
+        const uint32_t before = block_sum_1024(part, warp_sums);
+        // exclusive scan of this CTA's flags
+        const uint32_t flag = (b < B && mask[b] != 0) ? 1u : 0u;
+        uint32_t incl = flag;
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xffffffffu, incl, o);
+            if ((int)(threadIdx.x & 31) >= o) incl += up;
+        }
+        __syncthreads();
+        if ((threadIdx.x & 31) == 31) warp_sums[threadIdx.x >> 5] = incl;
+        __syncthreads();
+        uint32_t warps_before = 0;
+        for (int w = 0; w < (int)(threadIdx.x >> 5); ++w) warps_before += warp_sums[w];
+        const uint32_t at = before + warps_before + incl - flag;
+        if (b < B) {
+            pos[b] = at;
+            if (flag) olist[at] = (uint32_t)b;
         }
     }
 }

@@ -129,3 +129,21 @@ def test_misuse_is_reported():
     assert L.cser_wshard_message_elems(plain.h, 0) == -1
     assert not L.cser_create_wshard(1000, 5, 4, 10, 2, 2, 2, 0.1, 0.0, 0)    # n_local > n_total
     c.close(), plain.close()
+
+
+@pytest.mark.skipif(torch.cuda.device_count() < 2, reason="needs two GPUs")
+def test_two_ranks_on_two_gpus_with_an_nccl_all_reduce():
+    """The workers split over two processes on two GPUs, the packed message summed by NCCL: every rank's state
+    must match the oracle within the stated tolerances (the sum over workers is associated rank by rank)."""
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    env = {**os.environ, "NCCL_NVLS_ENABLE": "0"}
+    res = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
+                          "--master-addr", "127.0.0.1", "--master-port", str(port),
+                          os.path.join(root, "tests", "wshard_ranks_check.py")],
+                         capture_output=True, text=True, timeout=600, env=env)
+    assert res.returncode == 0 and "WSHARD_RANKS_OK" in res.stdout, res.stdout[-2000:] + res.stderr[-2000:]
