@@ -166,7 +166,10 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size,
                            float eta, float beta, uint64_t seed, int64_t block_begin,
                            uint32_t flags);
 
-/* Free everything the handle owns.  The caller must have synchronized its streams. NULL is ignored. */
+/*
+ * Free everything the handle owns (no passage of the paper: lifecycle).  The caller must have
+ * synchronized its streams; the library waits for its own auxiliary stream.  NULL is ignored.
+ */
 void cser_destroy(cser_handle h);
 
 /*
@@ -217,7 +220,8 @@ int cser_replay_end(cser_handle h, void *stream);
 int cser_step_host(cser_handle h, const float *grad_host, void *stream);
 
 /*
- * Copy one piece of state to dst (host or device), enqueued on `stream`.
+ * Copy one piece of state to dst (host or device), enqueued on `stream` (no passage of the paper:
+ * inspection and checkpointing of the state of Algorithm 2 / 4: x_i, e_i, m_i, the masks, t).
  * dst_bytes must be at least the size of the piece: n*d*4 for x/e/m, B for a mask,
  * 8 for t.  CSER_STATE_M with beta == 0 is CSER_ERR_INVALID.
  */
@@ -233,23 +237,34 @@ int cser_read_columns(cser_handle h, int which, int64_t col_begin, int64_t col_c
 
 /*
  * Learning rate eta for the following steps (the schedules of Section 5.1 change it between
- * steps; Algorithms 2 and 4 take it as given).  Takes effect with the next cser_step.
+ * steps; Algorithms 2 and 4 take it as given).  Takes effect with the next cser_step.  A step
+ * captured in a CUDA graph carries the eta of capture time: replays do not see a later change.
  */
 int cser_set_lr(cser_handle h, float eta);
 
 /*
  * Restore one piece of state from src (host or device) - the inverse of
- * cser_read_state, for checkpoint/resume.  `bytes` must be exactly the piece's size.
+ * cser_read_state, for checkpoint/resume (no passage of the paper: lifecycle).  `bytes` must be exactly the piece's size.
  * Masks cannot be written (use cser_debug_set_masks).
  */
 int cser_write_state(cser_handle h, int which, const void *src, size_t bytes, void *stream);
 
 /*
- * Test hook: the NEXT cser_step uses these block masks (uint8 [B] each, host or
+ * Test hook (no passage of the paper): the NEXT cser_step uses these block masks (uint8 [B] each, host or
  * device, non-zero = selected) instead of drawing them.  r_mask may be NULL if
  * that step is not a reset step.  The copy is enqueued on `stream`.
  */
 int cser_debug_set_masks(cser_handle h, const uint8_t *g_mask, const uint8_t *r_mask, void *stream);
+
+/*
+ * Test hook for the bounded waits of the CSER_FLAG_STAGED_SELECTED kernel (no passage of the paper).
+ * In the NEXT cser_step one CTA of that kernel is told to expect 16 bytes that no copy delivers, and every
+ * wait is limited to wait_mcycles million SM clock cycles (1 .. 2000; the normal limit is 2000, about a
+ * second).  The wait runs out, the CTA leaves, the kernel ends, and every later cser_step /
+ * cser_read_state on the handle returns CSER_ERR_CUDA.  The state is then incomplete: destroy the handle.
+ * Nothing traps and the CUDA context stays usable.
+ */
+int cser_debug_stall_next_staged_step(cser_handle h, unsigned wait_mcycles);
 
 /*
  * Stand-alone GRBS block-select kernel (Definition 2): writes uint8 flags of blocks
@@ -286,8 +301,8 @@ int cser_wshard_pack(cser_handle h, const float *grad, float *msg, size_t msg_el
 int cser_wshard_apply(cser_handle h, const float *msg, void *stream);
 
 /*
- * Per-kernel timing.  With on != 0, cser_step brackets its mask kernel and its
- * fused step kernel with CUDA events on the launching stream.
+ * Per-kernel timing (no passage of the paper: measurement).  With on != 0, cser_step brackets its
+ * mask kernel and its step kernels with CUDA events on the launching stream.
  * cser_last_kernel_ms waits for the last step's events and returns both durations
  * in milliseconds (either pointer may be NULL).
  */
@@ -339,7 +354,7 @@ int cser_step_noalloc(int64_t d, int32_t n_workers, int32_t block_size,
                       float eta, float beta, uint64_t seed, uint64_t t,
                       const float *grad, float *x, float *e, float *m, void *stream);
 
-/* Thread-local description of the last error in this thread ("" if none). */
+/* Thread-local description of the last error in this thread ("" if none).  No passage of the paper: error reporting. */
 const char *cser_last_error(void);
 
 #ifdef __cplusplus

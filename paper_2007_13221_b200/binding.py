@@ -75,6 +75,8 @@ def lib():
     L.cser_step_noalloc.argtypes = [c.c_int64, c.c_int32, c.c_int32, c.c_uint32, c.c_uint32, c.c_int32,
                                     c.c_float, c.c_float, c.c_uint64, c.c_uint64,
                                     c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+    L.cser_debug_stall_next_staged_step.restype = c.c_int
+    L.cser_debug_stall_next_staged_step.argtypes = [c.c_void_p, c.c_uint]
     L.cser_last_error.restype = c.c_char_p
     L.cser_last_error.argtypes = []
     for name in ("cser_set_x0", "cser_step", "cser_step_host", "cser_read_state", "cser_write_state",

@@ -118,6 +118,8 @@ struct cser_ctx {
     bool fused_small = true;                         // small problems as one launch (off with CSER_FLAG_THREE_KERNELS)
     int sm_count = 0;
     unsigned *err_host = nullptr, *err_dev = nullptr;
+    unsigned wait_mcycles = 2000;                    // about a second at 2 GHz
+    bool test_stall = false;                         // cser_debug_stall_next_staged_step
     float *x0_stage = nullptr;                       // [d] staging for a host x0
     bool masks_injected = false;
     bool vec4 = false;                               // 128-bit path usable for the state arrays
@@ -453,6 +455,7 @@ int launch_step(cser_ctx *h, const float *grad, long long col0, long long col1, 
     P.tiles = 0, P.rctl = nullptr;
     P.list_cap = (unsigned)h->B;
     P.chunk_cols = P.n_chunks = P.stages = 0, P.err_word = nullptr;
+    P.wait_mcycles = h->wait_mcycles, P.test_stall = h->test_stall ? 1u : 0u;
     P.mask_g_out = P.mask_r_out = nullptr, P.block_begin = h->block_begin;
     P.k0 = P.k1 = P.t_lo = P.t_hi = 0, P.R1 = h->R1, P.R2 = h->R2;
     P.d = h->d, P.n = h->n;
@@ -772,6 +775,7 @@ int cser_step(cser_handle h, const float *grad, void *stream) {
     if (!rc && !fused) rc = select_for_iteration(h, is_reset, s);
     if (!rc && h->timing && cudaEventRecord(h->ev[1], s) != cudaSuccess) rc = fail(CSER_ERR_CUDA, "cser_step: event record failed");
     if (!rc) rc = fused ? launch_fused_small(h, grad, is_reset, s) : launch_step(h, grad, 0, h->d, is_reset, s, true);
+    h->test_stall = false;
     if (rc) return abandon_iteration(h, t_before, rc);
     if (h->timing) {
         CU_TRY(cudaEventRecord(h->ev[2], s));
@@ -1164,6 +1168,15 @@ int cser_replay_end(cser_handle h, void *stream) {
         CU_TRY(cudaMemcpy(h->mask_r_half[1], h->sb[0].mask_r, (size_t)h->B, cudaMemcpyDeviceToDevice));
         h->mask_r = h->last_mask_r = h->mask_r_half[1];
     }
+    return CSER_OK;
+}
+
+int cser_debug_stall_next_staged_step(cser_handle h, unsigned wait_mcycles) {
+    if (int rc = check_handle(h)) return rc;
+    if (!h->staging) return fail(CSER_ERR_INVALID, "cser_debug_stall_next_staged_step: handle has no staged kernel");
+    if (wait_mcycles == 0 || wait_mcycles > 2000) return fail(CSER_ERR_INVALID, "wait_mcycles must be in 1 .. 2000");
+    h->wait_mcycles = wait_mcycles;
+    h->test_stall = true;
     return CSER_OK;
 }
 

@@ -104,6 +104,7 @@ __global__ void __launch_bounds__(kStagedThreads) cser_selected_staged_kernel(co
     const unsigned n = (unsigned)P.n;
     const size_t stage_bytes = (size_t)NA * n * C * 16u;
     const unsigned warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long wait_cycles = (long long)P.wait_mcycles * 1000000ll;
 
     if (threadIdx.x == 0) {
         for (unsigned s = 0; s < S; ++s) {
@@ -144,7 +145,7 @@ __global__ void __launch_bounds__(kStagedThreads) cser_selected_staged_kernel(co
             const unsigned blk = DENSE ? first_blk + (unsigned)entry : P.list[entry];
             const bool sg = P.mask_g[blk] != 0;
             const bool sr = reset_on ? (P.mask_r[blk] != 0) : false;
-            if (round > 0 && !mbar_wait_bounded(&ctl->empty[s], (round - 1) & 1u)) {
+            if (round > 0 && !mbar_wait_bounded(&ctl->empty[s], (round - 1) & 1u, wait_cycles)) {
                 ok = false;
                 break;
             }
@@ -162,7 +163,9 @@ __global__ void __launch_bounds__(kStagedThreads) cser_selected_staged_kernel(co
                 ctl->unit[s].c0 = lo;
                 ctl->unit[s].cols = cols;
                 ctl->unit[s].flags = (sg ? 1u : 0u) | (sr ? 2u : 0u);
-                if (cols) mbar_arrive_expect(&ctl->full[s], n_arr * n * cols * 16u);
+                // (test hook: bytes that never arrive make this unit's wait run out)
+                const uint32_t phantom = (P.test_stall && blockIdx.x == 0 && k == 0) ? 16u : 0u;
+                if (cols) mbar_arrive_expect(&ctl->full[s], n_arr * n * cols * 16u + phantom);
                 else      mbar_arrive(&ctl->full[s]);
             }
             __syncwarp();
@@ -188,7 +191,7 @@ __global__ void __launch_bounds__(kStagedThreads) cser_selected_staged_kernel(co
             // give the copies already issued a bounded time to land before the CTA's memory goes away
             const unsigned long long from = k > S ? k - S : 0ull;
             for (unsigned long long j = from; j < k; ++j)
-                mbar_wait_bounded(&ctl->full[j % S], (unsigned)(j / S) & 1u, kWaitCycles / 64);
+                mbar_wait_bounded(&ctl->full[j % S], (unsigned)(j / S) & 1u, wait_cycles / 64);
         }
         return;
     }
@@ -204,7 +207,7 @@ __global__ void __launch_bounds__(kStagedThreads) cser_selected_staged_kernel(co
     for (int q = 0; q < 4; ++q) zero.v[q] = 0.f;
     for (unsigned long long k = 0; k < n_my; ++k) {
         const unsigned s = (unsigned)(k % S);
-        const bool landed = mbar_wait_bounded(&ctl->full[s], (unsigned)(k / S) & 1u);
+        const bool landed = mbar_wait_bounded(&ctl->full[s], (unsigned)(k / S) & 1u, wait_cycles);
         if (!consumers_all(landed)) {
             if (!landed) staged_fail(P, 2u);
             return;

@@ -60,6 +60,8 @@ struct StepParams {
     unsigned n_chunks;       // work units per block
     unsigned stages;         // stages of the copy ring
     unsigned *err_word;      // host-visible word a wait that ran out raises (may be NULL)
+    unsigned wait_mcycles;   // limit of every barrier wait, in millions of SM clock cycles
+    unsigned test_stall;     // test hook: CTA 0 announces 16 bytes for its first unit that never arrive
     // single-launch kernel for small problems only (it draws the masks itself):
     uint8_t *mask_g_out, *mask_r_out;
     long long block_begin;   // global id of block 0

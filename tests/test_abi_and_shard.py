@@ -92,9 +92,6 @@ def _problem():
     return n, d, T, x0, g
 
 
-class _SlabOracle(CSEROracle):
-    """Oracle on a slab: same columns as a `cols` subset of the global vector."""
-
 
 def _run_slab(rank, world):
     n, d, T, x0, g = _problem()

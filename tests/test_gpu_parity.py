@@ -640,6 +640,46 @@ def test_step_captured_once_in_a_cuda_graph_and_replayed():
     opt.close()
 
 
+@pytest.mark.parametrize("n_plain,n_replay", [(3, 2), (2, 2), (4, 4), (1, 1)])
+def test_reset_mask_of_the_last_reset_step_stays_readable_around_replay_mode(n_plain, n_replay):
+    """CSER_STATE_MASK_R is the reset mask of the last reset step that was executed - also when replay mode
+    ends one step before a reset (its select kernel has then already prepared the next reset mask), when no
+    reset ran during replay, and on the ordinary steps that follow."""
+    d, n, bs, R1, R2, H = 4096 + 40, 4, 64, 4, 2, 3
+    rng = np.random.default_rng(3)
+    opt = b.CSER(d, n, bs, R1, R2, H, 0.1, 0.9, 17, flags=b.FLAG_THREE_KERNELS)
+    ref = CSEROracle(d, n, bs, R1, R2, H, 0.1, 0.9, 17, dtype=np.float32)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    opt.set_x0(torch.from_numpy(x0).to(DEV)), ref.set_x0(x0)
+    g = torch.empty((n, d), device=DEV)
+
+    def check(t):
+        if t >= H:
+            assert np.array_equal(opt.state(b.STATE_MASK_R).cpu().numpy(), ref.mask_r), t
+        assert np.array_equal(opt.state(b.STATE_X).cpu().numpy(), ref.x), t
+
+    t = 0
+    for _ in range(n_plain):
+        t += 1
+        g.copy_(torch.from_numpy(rng.standard_normal((n, d)).astype(np.float32)))
+        opt.step(g), ref.step(g.cpu().numpy())
+        check(t)
+    b.cser_replay_begin(opt.h)
+    for _ in range(n_replay):
+        t += 1
+        g.copy_(torch.from_numpy(rng.standard_normal((n, d)).astype(np.float32)))
+        b.cser_step_replayable(opt.h, g), ref.step(g.cpu().numpy())
+        check(t)
+    b.cser_replay_end(opt.h)
+    check(t)
+    for _ in range(4):
+        t += 1
+        g.copy_(torch.from_numpy(rng.standard_normal((n, d)).astype(np.float32)))
+        opt.step(g), ref.step(g.cpu().numpy())
+        check(t)
+    opt.close()
+
+
 # ------------------------------------------------------------------ randomized differential test
 def test_random_shapes_parameters_and_flags_against_the_float32_oracle():
     """400 random problems (shape, ratios, reset interval, momentum, flags, injected masks now and
@@ -749,6 +789,41 @@ def test_staged_kernel_with_injected_masks_replay_and_host_gradients():
     for which in (b.STATE_X, b.STATE_E, b.STATE_M):
         assert torch.equal(a.state(which), c.state(which)), which
     a.close(), c.close()
+
+
+def test_a_staged_kernel_wait_that_runs_out_is_reported_and_nothing_hangs():
+    """The staged kernel's waits on its shared-memory barriers are bounded.  One CTA is told to expect bytes
+    that never arrive (test hook) with the limit lowered to 0.1 s: the kernel must end by itself, the handle
+    must report the failure on every later call, and the CUDA context must stay usable (another handle steps
+    on, a plain copy works)."""
+    import time
+    L = b.lib()
+    d, n, bs = 64 * 300, 4, 64
+    bad = b.CSER(d, n, bs, 2, 2, 2, 0.1, 0.9, 3, flags=b.FLAG_STAGED_SELECTED)
+    good = b.CSER(d, n, bs, 2, 2, 2, 0.1, 0.9, 3, flags=b.FLAG_STAGED_SELECTED)
+    x0 = torch.randn(d, device=DEV)
+    bad.set_x0(x0), good.set_x0(x0)
+    g = torch.randn((n, d), device=DEV)
+    bad.step(g), good.step(g)
+    torch.cuda.synchronize()
+    assert L.cser_debug_stall_next_staged_step(bad.h, 200) == 0
+    t0 = time.perf_counter()
+    bad.step(g)                                        # enqueues the stalled kernel
+    torch.cuda.synchronize()                           # ... which ends by itself
+    assert time.perf_counter() - t0 < 10.0
+    assert L.cser_step(bad.h, ctypes.c_void_p(g.data_ptr()), None) == -3
+    assert "wait ran out" in b.cser_last_error()
+    out = torch.empty((n, d), device=DEV)
+    assert L.cser_read_state(bad.h, b.STATE_X, ctypes.c_void_p(out.data_ptr()), out.numel() * 4, None) == -3
+    good.step(g)                                       # the context is fine
+    torch.cuda.synchronize()
+    assert bool(torch.isfinite(good.state(b.STATE_X)).all())
+    assert torch.equal(g.clone(), g)
+    h = bad.h
+    bad.h = None
+    torch.cuda.synchronize()
+    b.cser_destroy(h)
+    good.close()
 
 
 # ------------------------------------------------------------------ C2 = 0 without an error array
