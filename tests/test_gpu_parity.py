@@ -972,3 +972,17 @@ def test_refused_steps_leave_the_counter_and_the_state_alone(launch_path):
     for which in (b.STATE_X, b.STATE_E, b.STATE_M, b.STATE_MASK_G, b.STATE_MASK_R):
         assert torch.equal(a.state(which), c.state(which)), which
     a.close(), c.close()
+
+
+@pytest.mark.skipif(torch.cuda.device_count() < 2, reason="needs a second GPU to own the foreign buffer")
+def test_a_buffer_of_another_gpu_is_refused_before_anything_is_launched():
+    """Device memory of another GPU passes a plain "is this device memory" check but would be dereferenced by
+    kernels of this GPU; it must be refused on the host (nothing is launched on it)."""
+    L = b.lib()
+    opt = b.CSER(1000, 2, 10, 2, 2, 2, 0.1, 0.0, 0)
+    foreign = torch.zeros((2, 1000), device="cuda:1")
+    torch.cuda.set_device(0)
+    assert L.cser_step(opt.h, ctypes.c_void_p(foreign.data_ptr()), None) == -1
+    assert "lives on device" in b.cser_last_error()
+    assert opt.t == 0
+    opt.close()
