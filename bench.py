@@ -532,15 +532,28 @@ def main():
 
     from paper_2007_13221_b200 import synth
     default_run = args.config == 0 and not args.d and args.R1 < 0 and args.R2 < 0 and args.H < 0
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    gpu_arm = args.impl == "ours" and args.oracle_slab < 0 and not args.ceilings
+    if gpu_arm:
+        import torch
+        import torch.distributed as dist
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+        torch.cuda.set_device(local)
+        if world > 1:
+            dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     if args.config == 0:
         args.config = HEADLINE_CONFIG
-        if args.impl == "ours":
-            import torch
+        if gpu_arm:
+            # the largest workload needs 53 GB per GPU; every rank must make the same choice
             need = synth.CONFIGS[HEADLINE_CONFIG].n_workers * synth.CONFIGS[HEADLINE_CONFIG].d * 4 * 5.3
-            if torch.cuda.is_available():
-                torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
-                if torch.cuda.mem_get_info()[0] < need:
-                    args.config = 2
+            fits = torch.tensor([1 if torch.cuda.mem_get_info()[0] >= need else 0], device=f"cuda:{local}")
+            if world > 1:
+                dist.all_reduce(fits, op=dist.ReduceOp.MIN)
+            if int(fits.item()) == 0:
+                args.config = 2
     w = synth.CONFIGS[args.config]
     if args.d:
         w = w.scaled(args.d)
@@ -559,18 +572,7 @@ def main():
         run_ceilings(args)
         return
 
-    import torch
-    import torch.distributed as dist
-
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
-    torch.cuda.set_device(local)
     dev = f"cuda:{local}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(dev))
     import __graft_entry__
     if rank == 0:
         __graft_entry__.build()
