@@ -218,7 +218,7 @@ def _cols_of(blocks, w):
     return np.concatenate(parts)
 
 
-def _full_size_parity(cfg, steps=None, n_random=192, impl2=False):
+def _full_size_parity(cfg, steps=None, n_random=192, impl2=False, flags=0):
     w = synth.CONFIGS[cfg]
     oracle = CSERImpl2Oracle if impl2 else CSEROracle
     steps = w.steps if steps is None else steps
@@ -232,7 +232,7 @@ def _full_size_parity(cfg, steps=None, n_random=192, impl2=False):
     refs = {dt: oracle(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
                        dtype=dt, cols=cols) for dt in (np.float32, np.float64)}
     opt = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, w.seed,
-                 flags=b.FLAG_NO_ERROR_ARRAY if impl2 else 0)
+                 flags=(b.FLAG_NO_ERROR_ARRAY if impl2 else 0) | flags)
     x0 = synth.x0(w, DEV)
     opt.set_x0(x0)
     x0_s = x0[cols_dev].cpu().numpy()
@@ -754,6 +754,13 @@ def test_staged_selected_block_kernel_equals_float32_oracle_exactly(d, n, bs, R1
         got, want = opt.state(which).cpu().numpy(), getattr(ref, name)
         assert np.array_equal(got, want), (name, int((got != want).sum()))
     opt.close()
+
+
+@pytest.mark.parametrize("cfg", [2, 3])
+def test_staged_kernel_full_size_on_sampled_blocks(cfg):
+    """The opt-in staged kernel at full size in the launch configuration `bench.py --staged` times: the
+    WRN-sized workload (blocks in one chunk) and the ResNet-50-sized one (n = 16: blocks cut into chunks)."""
+    _full_size_parity(cfg, steps=16, flags=b.FLAG_STAGED_SELECTED)
 
 
 def test_staged_kernel_with_injected_masks_replay_and_host_gradients():
