@@ -922,6 +922,36 @@ def test_checkpoint_and_resume_is_bit_identical(launch_path):
     a.close(), c.close()
 
 
+def test_step_counter_across_the_32_bit_boundary(launch_path):
+    """t is a 64-bit counter and enters the Philox counter as two 32-bit words: steps t = 2^32 - 1 .. 2^32 + 3
+    (the counter restored with cser_write_state) must draw the oracle's masks and give its state, on both
+    launch paths and in replay mode."""
+    d, n, bs, R1, R2, H = 4096 + 40, 4, 64, 4, 2, 2
+    t0 = 2**32 - 2
+    rng = np.random.default_rng(11)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    opt = b.CSER(d, n, bs, R1, R2, H, 0.1, 0.9, 5)
+    ref = CSEROracle(d, n, bs, R1, R2, H, 0.1, 0.9, 5, dtype=np.float32)
+    opt.set_x0(torch.from_numpy(x0).to(DEV)), ref.set_x0(x0)
+    b.cser_write_state(opt.h, b.STATE_T, torch.tensor([t0], dtype=torch.int64))
+    ref.t = t0
+    for k in range(1, 8):
+        g = rng.standard_normal((n, d)).astype(np.float32)
+        gd = torch.from_numpy(g).to(DEV)
+        if k == 5:
+            b.cser_replay_begin(opt.h)
+            b.cser_step_replayable(opt.h, gd)
+            b.cser_replay_end(opt.h)
+        else:
+            opt.step(gd)
+        ref.step(g)
+        assert opt.t == t0 + k
+        assert np.array_equal(opt.state(b.STATE_MASK_G).cpu().numpy(), ref.mask_g), k
+    for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e"), (b.STATE_M, "m")):
+        assert np.array_equal(opt.state(which).cpu().numpy(), getattr(ref, name)), name
+    opt.close()
+
+
 def test_errors_are_reported_not_raised_on_the_device():
     L = b.lib()
     assert not L.cser_create(0, 8, 256, 4, 4, 4, 0.1, 0.0, 0)
