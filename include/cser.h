@@ -150,15 +150,18 @@ cser_handle cser_create_slab(int64_t d, int32_t n_workers, int32_t block_size,
  */
 #define CSER_FLAG_STAGED_SELECTED 8u
 /*
- *   CSER_FLAG_THREE_KERNELS  an iteration is normally three kernels (block select, streaming kernel
- *       for the unselected blocks, selected-block kernel beside it).  When an iteration moves at most
- *       256 MB (n_workers * d * 28 bytes with momentum and an error array) it would take a few tens
- *       of microseconds and the kernel boundaries would cost as much as the traffic, so cser_step
- *       runs it as ONE kernel instead, which draws the masks
- *       itself (same Philox draws, same arithmetic, bit-identical results).  This flag keeps the
- *       three kernels at every size.  Steps with injected masks, exact-count masks, replayable steps,
- *       cser_step_host and vectors whose d or block_size is not a multiple of 4 use the three
- *       kernels in any case.
+ *   CSER_FLAG_THREE_KERNELS  an iteration of a large problem is three kernels (block select, streaming
+ *       kernel for the unselected blocks, selected-block kernel beside it).  cser_step runs an iteration
+ *       as ONE kernel instead, which draws the masks itself and walks every column over the workers
+ *       (same Philox draws, same arithmetic, bit-identical results), in two cases: when the iteration
+ *       moves at most 256 MB (n_workers * d * 28 bytes with momentum and an error array), because it
+ *       would take a few tens of microseconds and the kernel boundaries would cost as much as the
+ *       traffic; and, with at most 8 workers, when a large share of the blocks is selected in that
+ *       iteration (1/R1 >= 1/4 on an ordinary step, 1/R1 + 1/R2 >= 1/10 on a reset step), because walking
+ *       all columns in their natural order then beats sending scattered blocks through the selected-block
+ *       kernel.  This flag keeps the three kernels for every iteration.  Steps with injected masks,
+ *       exact-count masks, replayable steps, cser_step_host and vectors whose d or block_size is not a
+ *       multiple of 4 use the three kernels in any case.
  */
 #define CSER_FLAG_THREE_KERNELS 16u
 cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size,

@@ -233,9 +233,36 @@ int select_for_iteration(cser_ctx *h, bool is_reset, cudaStream_t s) {
 // kernel boundaries, events and stream waits of the three-kernel step cost more than its better use
 // of DRAM gains (about 10 us against 8 % of the traffic time; the two designs were measured to break
 // even at 235 to 300 MB per step).
-constexpr long long kFusedMaxBytes = 1ll << 28;
+#ifndef CSER_FUSED_MAX_BYTES
+#define CSER_FUSED_MAX_BYTES (1ll << 28)
+#endif
+constexpr long long kFusedMaxBytes = CSER_FUSED_MAX_BYTES;
 long long step_bytes_bound(const cser_ctx *h) {
     return (long long)h->n * h->d * (12 + (h->m ? 8 : 0) + (h->e ? 8 : 0));
+}
+// The same kernel also wins on large problems when a large share of the blocks is selected: there the
+// three-kernel step sends that share through the selected-block kernel as scattered pieces of one block
+// per worker, while the single-launch kernel walks all columns in their natural order.  Measured on the
+// WRN-40-8-sized vector (n = 8; ordinary / reset steps in ms, three kernels against one launch): R = 2
+// 1.113 / 1.526 against 1.077 / 1.179; R = 4 1.165 / 1.449 against 1.164 / 1.196; R = 8 1.179 / 1.338
+// against 1.206 / 1.219; R = 16 1.177 / 1.256 against 1.226 / 1.233; R = 32 1.178 / 1.226 against
+// 1.237 / 1.242.  Hence one launch from a selected share of 1/4 on ordinary steps and of 1/10 on reset
+// steps (update mask and reset mask together), for up to 8 workers (with 16 the walk over all
+// columns loses more than it gains).
+#ifndef CSER_FUSED_SHARE_PLAIN
+#define CSER_FUSED_SHARE_PLAIN 0.25
+#define CSER_FUSED_SHARE_RESET 0.10
+#define CSER_FUSED_SHARE_MAX_WORKERS 8
+#endif
+// Whether iteration number t of handle h goes through the single-launch kernel (given a gradient
+// pointer that allows 128-bit loads).
+bool fused_for_iteration(const cser_ctx *h, uint64_t t) {
+    if (!(h->fused_small && h->vec4 && !h->exact && !h->replay && h->n_total == 0 && h->n_buf == 2)) return false;
+    if (step_bytes_bound(h) <= kFusedMaxBytes) return true;
+    if (h->n > CSER_FUSED_SHARE_MAX_WORKERS || h->d / 4 > 0xffffffffll) return false;
+    const bool is_reset = (t % (uint64_t)h->H) == 0;
+    const double share = (h->R1 ? 1.0 / h->R1 : 0.0) + (is_reset ? 1.0 / h->R2 : 0.0);
+    return share >= (is_reset ? CSER_FUSED_SHARE_RESET : CSER_FUSED_SHARE_PLAIN);
 }
 
 // Work-unit geometry of the staged selected-block kernel: C vector columns per unit so that all n
@@ -320,8 +347,7 @@ int launch_step_v(cser_ctx *h, const StepParams &P, bool is_reset, cudaStream_t 
     const bool have_aux = use_aux && h->aux != nullptr && h->n_total == 0;
     const bool beside = have_aux && stream_any;                       // selected-block kernel beside the streaming one
     // next iteration's select kernel on aux (not where the single-launch kernel will run that iteration)
-    const bool prefetch = have_aux && !h->replay && h->n_buf == 2 &&
-                          !(h->fused_small && h->vec4 && !h->exact && step_bytes_bound(h) <= kFusedMaxBytes);
+    const bool prefetch = have_aux && !h->replay && h->n_buf == 2 && !fused_for_iteration(h, h->t + 1);
     const bool fork = beside || prefetch;
     if (fork) {
         CU_TRY(cudaEventRecord(h->ev_fork, s));
@@ -473,8 +499,7 @@ int launch_step(cser_ctx *h, const float *grad, long long col0, long long col1, 
 }
 
 bool fused_applies(const cser_ctx *h, const float *grad) {
-    return h->fused_small && h->vec4 && !h->exact && !h->masks_injected && !h->replay && h->n_total == 0 &&
-           (uintptr_t)grad % 16 == 0 && step_bytes_bound(h) <= kFusedMaxBytes;
+    return !h->masks_injected && (uintptr_t)grad % 16 == 0 && fused_for_iteration(h, h->t);
 }
 
 // The whole iteration h->t in one launch (small problems): masks drawn inside the kernel and recorded
@@ -511,12 +536,27 @@ int launch_fused_small(cser_ctx *h, const float *grad, bool is_reset, cudaStream
         if (err) kernel = is_reset ? cser_fused_small_kernel<false, true, true> : cser_fused_small_kernel<false, false, true>;
         else     kernel = is_reset ? cser_fused_small_kernel<false, true, false> : cser_fused_small_kernel<false, false, false>;
     }
+    // if the next iteration takes the three kernels, its select kernel runs beside this kernel
+    const bool prefetch = h->aux != nullptr && !fused_for_iteration(h, h->t + 1);
+    if (prefetch) {
+        CU_TRY(cudaEventRecord(h->ev_fork, s));
+        CU_TRY(cudaStreamWaitEvent(h->aux, h->ev_fork, 0));
+    }
     CU_TRY(cudaLaunchKernelEx(&cfg, kernel, P));
     h->launches++;
+    h->pre_valid = false;
+    if (prefetch) {
+        const uint64_t t_next = h->t + 1;
+        const int rc = launch_select(h, h->cur ^ 1, t_next, (t_next % (uint64_t)h->H) == 0, true, h->aux,
+                                     &h->pre_count);
+        h->pre_valid = rc == CSER_OK;
+        h->pre_t = t_next;
+        CU_TRY(cudaEventRecord(h->ev_pre, h->aux));
+        h->pre_pending = true;
+    }
     // what activate_selection does for the three-kernel step
     h->mask_g = h->sb[h->cur].mask_g, h->sel_list = h->sb[h->cur].list;
     if (is_reset) h->mask_r = h->last_mask_r = reset_mask_of(h, h->t);
-    h->pre_valid = false;
     h->walk_all = false;
     return CSER_OK;
 }

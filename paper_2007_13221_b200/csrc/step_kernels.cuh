@@ -344,10 +344,11 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
 // selected-block kernel, unselected ones elementwise (x_i -= p_i, e_i -= p_i).
 template <bool MOM, bool RESET, bool ERR>
 __global__ void __launch_bounds__(kWalkThreads) cser_fused_small_kernel(const StepParams P) {
-    // (measured on the d = 2^20, n = 8 workload: 1 / 2 / 4 / 8 workers in flight give 54.7k / 59.2k / 59.1k /
-    // 47.1k steps/s)
+    // (measured: on the d = 2^20, n = 8 workload 1 / 2 / 4 / 8 workers in flight give 54.7k / 59.2k / 59.1k /
+    // 47.1k steps/s; on the WRN-40-8-sized vector with R = 2, 4 workers in flight give 921 steps/s against
+    // 902 with 2)
 #ifndef CSER_FUSED_U
-#define CSER_FUSED_U 2
+#define CSER_FUSED_U 4
 #endif
     constexpr int V = 4, U = CSER_FUSED_U;   // workers whose loads are in flight together on an unselected block
     const long long c = (long long)blockIdx.x * kWalkThreads + threadIdx.x;

@@ -727,6 +727,21 @@ def test_random_shapes_parameters_and_flags_against_the_float32_oracle():
         opt.close()
 
 
+@pytest.mark.parametrize("R1,R2,H", [(16, 16, 2), (4, 4, 3), (16, 2, 2), (64, 64, 2)])
+def test_large_problems_switch_between_one_launch_and_three_kernels_step_by_step(R1, R2, H):
+    """Above 256 MB per step the launch path is chosen per iteration from the expected share of selected
+    blocks (one launch from 1/4 on ordinary steps and from 1/10 on reset steps): (16, 16) and (16, 2)
+    alternate between the paths, (4, 4) is all one launch, (64, 64) all three kernels.  Whatever the mix, masks
+    and state must equal the float32 oracle's, and the reset mask must stay readable."""
+    d, n, bs = 1_300_000 + 4, 8, 512
+    assert n * d * 28 > 1 << 28
+    opt, ref = _run_both(d, n, bs, R1, R2, H, 0.1, 0.9, steps=7)
+    for which, name in ((b.STATE_X, "x"), (b.STATE_E, "e"), (b.STATE_M, "m")):
+        got, want = opt.state(which).cpu().numpy(), getattr(ref, name)
+        assert np.array_equal(got, want), (name, int((got != want).sum()))
+    opt.close()
+
+
 # ------------------------------------------------------------------ the opt-in staged selected-block kernel
 STAGED_SHAPES = [
     # d, n, bs, R1, R2, H, beta, flags
