@@ -516,7 +516,7 @@ int launch_fused_small(cser_ctx *h, const float *grad, bool is_reset, cudaStream
     P.t_lo = (uint32_t)(h->t & 0xffffffffu), P.t_hi = (uint32_t)(h->t >> 32);
     P.mask_g_out = h->sb[h->cur].mask_g;
     P.mask_r_out = reset_mask_of(h, h->t);
-    const unsigned grid = (unsigned)((P.cols_total + kWalkThreads - 1) / kWalkThreads);
+    const unsigned grid = (unsigned)((P.cols_total + kFusedThreads - 1) / kFusedThreads);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeAccessPolicyWindow;
     attr[0].val.accessPolicyWindow.base_ptr = h->state_base;
@@ -525,7 +525,7 @@ int launch_fused_small(cser_ctx *h, const float *grad, bool is_reset, cudaStream
     attr[0].val.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
     attr[0].val.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid), cfg.blockDim = dim3(kWalkThreads), cfg.dynamicSmemBytes = 0, cfg.stream = s;
+    cfg.gridDim = dim3(grid), cfg.blockDim = dim3(kFusedThreads), cfg.dynamicSmemBytes = 0, cfg.stream = s;
     cfg.attrs = attr, cfg.numAttrs = h->l2_persist ? 1 : 0;
     const bool mom = h->m != nullptr, err = h->e != nullptr;
     void (*kernel)(const StepParams);

@@ -342,8 +342,14 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
 // operations, which is cheaper than a kernel boundary), the first thread of each block records them
 // for cser_read_state, and the column is then walked over the workers: selected blocks as in the
 // selected-block kernel, unselected ones elementwise (x_i -= p_i, e_i -= p_i).
+// CTA width: 64 / 128 / 256 / 512 threads were measured; 128 is best or within 1 % of best on the small
+// workload (59.1k steps/s against 54.5k at 256) and on the WRN-40-8-sized vector with R = 1, 2, 4.
+#ifndef CSER_FUSED_THREADS
+#define CSER_FUSED_THREADS 128
+#endif
+constexpr int kFusedThreads = CSER_FUSED_THREADS;
 template <bool MOM, bool RESET, bool ERR>
-__global__ void __launch_bounds__(kWalkThreads) cser_fused_small_kernel(const StepParams P) {
+__global__ void __launch_bounds__(kFusedThreads) cser_fused_small_kernel(const StepParams P) {
     // (measured: on the d = 2^20, n = 8 workload 1 / 2 / 4 / 8 workers in flight give 54.7k / 59.2k / 59.1k /
     // 47.1k steps/s; on the WRN-40-8-sized vector with R = 2, 4 workers in flight give 921 steps/s against
     // 902 with 2)
@@ -351,7 +357,7 @@ __global__ void __launch_bounds__(kWalkThreads) cser_fused_small_kernel(const St
 #define CSER_FUSED_U 4
 #endif
     constexpr int V = 4, U = CSER_FUSED_U;   // workers whose loads are in flight together on an unselected block
-    const long long c = (long long)blockIdx.x * kWalkThreads + threadIdx.x;
+    const long long c = (long long)blockIdx.x * kFusedThreads + threadIdx.x;
     if (c >= P.cols_total) return;
     const unsigned blk = (uint32_t)c / P.bsv;
     const uint32_t gb = (uint32_t)(P.block_begin + blk);
