@@ -206,7 +206,9 @@ int cser_step(cser_handle h, const float *grad, void *stream);
  * cser_step_host, cser_set_x0, cser_write_state and cser_debug_set_masks are refused;
  * cser_read_state works (the step counter is read from the device).  Not available with
  * exact-count masks or worker-sharded handles.  grad must be the same pointer at replay time
- * as at capture time (a captured launch carries its arguments).
+ * as at capture time (a captured launch carries its arguments).  A handle whose iterations move
+ * at most 256 MB replays as ONE kernel per step (see CSER_FLAG_THREE_KERNELS); it then needs a
+ * 16-byte aligned grad.
  */
 int cser_replay_begin(cser_handle h, void *stream);
 int cser_step_replayable(cser_handle h, const float *grad, void *stream);

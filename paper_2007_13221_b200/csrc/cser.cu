@@ -92,6 +92,7 @@ struct cser_ctx {
     // replayable steps (cser_replay_begin .. cser_replay_end): the iteration lives on the device
     ReplayCtl *ctl = nullptr;
     bool replay = false;
+    bool replay_fused = false;                       // replayable steps go through the single-launch kernel
     // worker-sharded mode (cser_create_wshard): n = local workers, n_total = all ranks' workers
     int n_total = 0;
     // ordered lists of the selected blocks, one set per mask buffer set (allocations of 2 B entries)
@@ -504,7 +505,7 @@ bool fused_applies(const cser_ctx *h, const float *grad) {
 
 // The whole iteration h->t in one launch (small problems): masks drawn inside the kernel and recorded
 // in the current buffer set.
-int launch_fused_small(cser_ctx *h, const float *grad, bool is_reset, cudaStream_t s) {
+int launch_fused_small(cser_ctx *h, const float *grad, bool is_reset, cudaStream_t s, bool replay = false) {
     if (int rc = join_prefetch(h, s)) return rc;       // a select kernel of an earlier three-kernel step
     StepParams P = {};
     P.g = grad, P.x = h->x, P.e = h->e, P.m = h->m;
@@ -516,6 +517,14 @@ int launch_fused_small(cser_ctx *h, const float *grad, bool is_reset, cudaStream
     P.t_lo = (uint32_t)(h->t & 0xffffffffu), P.t_hi = (uint32_t)(h->t >> 32);
     P.mask_g_out = h->sb[h->cur].mask_g;
     P.mask_r_out = reset_mask_of(h, h->t);
+    P.H = (uint32_t)h->H;
+    if (replay) {
+        // the kernel reads the iteration number from the device, decides there whether it resets, and
+        // records the masks in buffer set 0 (where cser_read_state looks in replay mode)
+        P.rctl = h->ctl;
+        P.mask_g_out = h->sb[0].mask_g, P.mask_r_out = h->sb[0].mask_r;
+        is_reset = true;
+    }
     const unsigned grid = (unsigned)((P.cols_total + kFusedThreads - 1) / kFusedThreads);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeAccessPolicyWindow;
@@ -537,7 +546,7 @@ int launch_fused_small(cser_ctx *h, const float *grad, bool is_reset, cudaStream
         else     kernel = is_reset ? cser_fused_small_kernel<false, true, false> : cser_fused_small_kernel<false, false, false>;
     }
     // if the next iteration takes the three kernels, its select kernel runs beside this kernel
-    const bool prefetch = h->aux != nullptr && !fused_for_iteration(h, h->t + 1);
+    const bool prefetch = !replay && h->aux != nullptr && !fused_for_iteration(h, h->t + 1);
     if (prefetch) {
         CU_TRY(cudaEventRecord(h->ev_fork, s));
         CU_TRY(cudaStreamWaitEvent(h->aux, h->ev_fork, 0));
@@ -554,6 +563,7 @@ int launch_fused_small(cser_ctx *h, const float *grad, bool is_reset, cudaStream
         CU_TRY(cudaEventRecord(h->ev_pre, h->aux));
         h->pre_pending = true;
     }
+    if (replay) return CSER_OK;
     // what activate_selection does for the three-kernel step
     h->mask_g = h->sb[h->cur].mask_g, h->sel_list = h->sb[h->cur].list;
     if (is_reset) h->mask_r = h->last_mask_r = reset_mask_of(h, h->t);
@@ -1160,13 +1170,19 @@ int cser_replay_begin(cser_handle h, void *stream) {
     c.c[0].t = h->t;           // block 0 stands for the iteration already done
     CU_TRY(cudaMemcpyAsync(h->ctl, &c, sizeof(c), cudaMemcpyHostToDevice, s));
     CU_TRY(cudaStreamSynchronize(s));   // c is on this function's stack
-    // masks and list of iteration t + 1 into buffer set 1, published in block 1
-    const unsigned grid = (unsigned)((h->B + 255) / 256);
-    grbs_select_replay_kernel<<<grid, 256, 0, s>>>(h->ctl, h->sb[0].mask_g, h->sb[0].mask_r, h->sb[0].list, h->Bpad,
-                                                   h->B, h->block_begin, (uint32_t)(h->seed & 0xffffffffu),
-                                                   (uint32_t)(h->seed >> 32), h->R1, h->R2, (uint32_t)h->H);
-    h->launches++;
-    CU_TRY(cudaGetLastError());
+    // Small problems replay as one launch per step (the kernel draws its masks itself); the choice is made
+    // once, here, because the two replay protocols keep different things in the control block.
+    h->replay_fused = h->fused_small && h->vec4 && step_bytes_bound(h) <= kFusedMaxBytes;
+    if (!h->replay_fused) {
+        // masks and list of iteration t + 1 into buffer set 1, published in block 1
+        const unsigned grid = (unsigned)((h->B + 255) / 256);
+        grbs_select_replay_kernel<<<grid, 256, 0, s>>>(h->ctl, h->sb[0].mask_g, h->sb[0].mask_r, h->sb[0].list,
+                                                       h->Bpad, h->B, h->block_begin,
+                                                       (uint32_t)(h->seed & 0xffffffffu), (uint32_t)(h->seed >> 32),
+                                                       h->R1, h->R2, (uint32_t)h->H);
+        h->launches++;
+        CU_TRY(cudaGetLastError());
+    }
     h->pre_valid = false;
     h->walk_all = false;
     h->replay = true;
@@ -1180,6 +1196,12 @@ int cser_step_replayable(cser_handle h, const float *grad, void *stream) {
     if (int rc = check_device_ptr(grad, "cser_step_replayable: grad")) return rc;
     if ((uintptr_t)grad % 4 != 0) return fail(CSER_ERR_INVALID, "cser_step_replayable: grad is not 4-byte aligned");
     cudaStream_t s = (cudaStream_t)stream;
+    if (h->replay_fused) {
+        if ((uintptr_t)grad % 16 != 0)
+            return fail(CSER_ERR_INVALID, "cser_step_replayable: this handle replays as one launch per step, "
+                                          "which needs a 16-byte aligned grad");
+        return launch_fused_small(h, grad, true, s, true);
+    }
     // the iteration prepared during the last step becomes the current one
     replay_advance_kernel<<<(unsigned)((h->B + 255) / 256), 256, 0, s>>>(h->ctl, h->sb[0].mask_g, h->sb[0].mask_r,
                                                                          h->sb[0].list, h->Bpad, h->B);

@@ -47,7 +47,7 @@ struct StepParams {
     const uint8_t *mask_g, *mask_r;
     const uint32_t *list;    // blocks selected by either mask this step
     const uint32_t *count;   // how many
-    const ReplayCtl *rctl;   // replayable steps: reset flag and list length are read on the device (else NULL)
+    ReplayCtl *rctl;         // replayable steps: iteration, reset flag and list length live on the device (else NULL)
     long long d;             // elements per row
     long long cols_total;    // vector columns per row
     long long c_begin;       // first vector column handled by this launch
@@ -66,6 +66,7 @@ struct StepParams {
     uint8_t *mask_g_out, *mask_r_out;
     long long block_begin;   // global id of block 0
     uint32_t k0, k1, t_lo, t_hi, R1, R2;
+    uint32_t H;              // reset interval (replayable single-launch steps decide on the device)
     int n;
     float eta, beta, n_f;
 };
@@ -348,64 +349,91 @@ __global__ void __launch_bounds__(kWalkThreads) cser_selected_kernel(const StepP
 #define CSER_FUSED_THREADS 128
 #endif
 constexpr int kFusedThreads = CSER_FUSED_THREADS;
-template <bool MOM, bool RESET, bool ERR>
-__global__ void __launch_bounds__(kFusedThreads) cser_fused_small_kernel(const StepParams P) {
-    // (measured: on the d = 2^20, n = 8 workload 1 / 2 / 4 / 8 workers in flight give 54.7k / 59.2k / 59.1k /
-    // 47.1k steps/s; on the WRN-40-8-sized vector with R = 2, 4 workers in flight give 921 steps/s against
-    // 902 with 2)
+// Workers whose loads are in flight together on an unselected block.  Measured: on the d = 2^20, n = 8
+// workload 1 / 2 / 4 / 8 give 54.7k / 59.2k / 59.1k / 47.1k steps/s; on the WRN-40-8-sized vector with R = 2,
+// 4 give 921 steps/s against 902 with 2.
 #ifndef CSER_FUSED_U
 #define CSER_FUSED_U 4
 #endif
-    constexpr int V = 4, U = CSER_FUSED_U;   // workers whose loads are in flight together on an unselected block
+template <bool MOM, bool RESET, bool ERR>
+__global__ void __launch_bounds__(kFusedThreads) cser_fused_small_kernel(const StepParams P) {
+    constexpr int V = 4, U = CSER_FUSED_U;
+    // Replayable steps (P.rctl set; the RESET variant is used): the iteration number lives on the device.
+    // Block c[0] holds the last iteration done; every CTA reads it, and the last CTA to finish writes it.
+    uint32_t t_lo = P.t_lo, t_hi = P.t_hi;
+    bool reset_on = RESET;
+    unsigned long long t_dev = 0;
+    if (P.rctl) {
+        t_dev = P.rctl->c[0].t + 1ull;
+        t_lo = (uint32_t)(t_dev & 0xffffffffu), t_hi = (uint32_t)(t_dev >> 32);
+        reset_on = RESET && (t_dev % P.H) == 0;
+    }
     const long long c = (long long)blockIdx.x * kFusedThreads + threadIdx.x;
-    if (c >= P.cols_total) return;
-    const unsigned blk = (uint32_t)c / P.bsv;
-    const uint32_t gb = (uint32_t)(P.block_begin + blk);
-    bool sg = false, sr = false;
-    if (P.R1 != 0)
-        sg = (unsigned long long)philox4x32_10_word0(P.k0, P.k1, gb, P.t_lo, P.t_hi, 0u) * P.R1 < (1ull << 32);
-    if constexpr (RESET)
-        sr = (unsigned long long)philox4x32_10_word0(P.k0, P.k1, gb, P.t_lo, P.t_hi, 1u) * P.R2 < (1ull << 32);
-    if (c == (long long)blk * P.bsv) {
-        P.mask_g_out[blk] = sg ? 1 : 0;
-        if constexpr (RESET) P.mask_r_out[blk] = sr ? 1 : 0;
-    }
-    if (sg || sr) {
-        walk_selected_column<V, MOM, RESET, ERR>(P, c, sg, sr);
-        return;
-    }
-    // C(p) = 0 on this block, so p' = r = p (Algorithm 3 lines 4-8): x_i -= p_i, e_i -= p_i
-    const long long d = P.d;
-    const int n = P.n;
-    const float *__restrict__ g = P.g + c * V;
-    float *__restrict__ x = P.x + c * V;
-    float *__restrict__ e = ERR ? P.e + c * V : nullptr;
-    float *__restrict__ m = MOM ? P.m + c * V : nullptr;
-    for (int i0 = 0; i0 < n; i0 += U) {
-        Pack<V> gv[U], mv[U], xv[U], ev[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            if (i0 + u < n) {
-                const long long o = (long long)(i0 + u) * d;
-                gv[u] = ld_stream<V>(g + o);
-                if constexpr (MOM) mv[u] = ld<V>(m + o);
-                xv[u] = ld<V>(x + o);
-                if constexpr (ERR) ev[u] = ld<V>(e + o);
+    if (c < P.cols_total) {
+        const unsigned blk = (uint32_t)c / P.bsv;
+        const uint32_t gb = (uint32_t)(P.block_begin + blk);
+        bool sg = false, sr = false;
+        if (P.R1 != 0)
+            sg = (unsigned long long)philox4x32_10_word0(P.k0, P.k1, gb, t_lo, t_hi, 0u) * P.R1 < (1ull << 32);
+        if constexpr (RESET) {
+            if (reset_on)
+                sr = (unsigned long long)philox4x32_10_word0(P.k0, P.k1, gb, t_lo, t_hi, 1u) * P.R2 < (1ull << 32);
+        }
+        if (c == (long long)blk * P.bsv) {
+            P.mask_g_out[blk] = sg ? 1 : 0;
+            if constexpr (RESET) {
+                if (reset_on) P.mask_r_out[blk] = sr ? 1 : 0;
             }
         }
+        if (sg || sr) {
+            walk_selected_column<V, MOM, RESET, ERR>(P, c, sg, sr);
+        } else {
+            // C(p) = 0 on this block, so p' = r = p (Algorithm 3 lines 4-8): x_i -= p_i, e_i -= p_i
+            const long long d = P.d;
+            const int n = P.n;
+            const float *__restrict__ g = P.g + c * V;
+            float *__restrict__ x = P.x + c * V;
+            float *__restrict__ e = ERR ? P.e + c * V : nullptr;
+            float *__restrict__ m = MOM ? P.m + c * V : nullptr;
+            for (int i0 = 0; i0 < n; i0 += U) {
+                Pack<V> gv[U], mv[U], xv[U], ev[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            if (i0 + u < n) {
-                const long long o = (long long)(i0 + u) * d;
-                const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], P.eta, P.beta);
-#pragma unroll
-                for (int k = 0; k < V; ++k) {
-                    xv[u].v[k] = xv[u].v[k] - p.v[k];
-                    if constexpr (ERR) ev[u].v[k] = ev[u].v[k] - p.v[k];
+                for (int u = 0; u < U; ++u) {
+                    if (i0 + u < n) {
+                        const long long o = (long long)(i0 + u) * d;
+                        gv[u] = ld_stream<V>(g + o);
+                        if constexpr (MOM) mv[u] = ld<V>(m + o);
+                        xv[u] = ld<V>(x + o);
+                        if constexpr (ERR) ev[u] = ld<V>(e + o);
+                    }
                 }
-                if constexpr (MOM) st<V>(m + o, mv[u]);
-                st<V>(x + o, xv[u]);
-                if constexpr (ERR) st<V>(e + o, ev[u]);
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    if (i0 + u < n) {
+                        const long long o = (long long)(i0 + u) * d;
+                        const Pack<V> p = get_p<V, MOM>(gv[u], mv[u], P.eta, P.beta);
+#pragma unroll
+                        for (int k = 0; k < V; ++k) {
+                            xv[u].v[k] = xv[u].v[k] - p.v[k];
+                            if constexpr (ERR) ev[u].v[k] = ev[u].v[k] - p.v[k];
+                        }
+                        if constexpr (MOM) st<V>(m + o, mv[u]);
+                        st<V>(x + o, xv[u]);
+                        if constexpr (ERR) st<V>(e + o, ev[u]);
+                    }
+                }
+            }
+        }
+    }
+    if (P.rctl) {
+        // a counter, no waiting: whoever finishes last moves the iteration number on
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            __threadfence();
+            if (atomicAdd(&P.rctl->c[0].done, 1u) == gridDim.x - 1) {
+                P.rctl->c[0].t = t_dev;
+                P.rctl->c[0].reset = reset_on ? 1u : 0u;
+                P.rctl->c[0].done = 0;
             }
         }
     }

@@ -574,7 +574,7 @@ def test_misaligned_gradient_pointer_takes_the_scalar_path():
 @pytest.mark.parametrize("d,n,bs,R1,R2,H,beta,flags", [
     (4096 + 40, 8, 256, 4, 2, 3, 0.9, 0), (1001, 3, 7, 2, 3, 2, 0.0, 0), (50_000, 16, 512, 8, 4, 1, 0.9, 0),
     (20_000, 4, 64, 1, 2, 4, 0.9, 0), (30_000, 8, 128, 0, 2, 2, 0.0, 0), (30_000, 8, 128, 4, 4, 2, 0.9, 1)])
-def test_replayable_steps_equal_ordinary_steps_and_the_oracle(d, n, bs, R1, R2, H, beta, flags):
+def test_replayable_steps_equal_ordinary_steps_and_the_oracle(d, n, bs, R1, R2, H, beta, flags, launch_path):
     """cser_step, then replayable steps (not captured), then cser_step again: one trajectory."""
     rng = np.random.default_rng(77)
     x0 = rng.standard_normal(d).astype(np.float32)
@@ -604,7 +604,7 @@ def test_replayable_steps_equal_ordinary_steps_and_the_oracle(d, n, bs, R1, R2, 
     opt.close()
 
 
-def test_step_captured_once_in_a_cuda_graph_and_replayed():
+def test_step_captured_once_in_a_cuda_graph_and_replayed(launch_path):
     w = synth.CONFIGS[2].scaled(d=400_000 + 8, steps=20)
     R1, R2, H = 4, 2, 3
     opt = b.CSER(w.d, w.n_workers, w.block_size, R1, R2, H, w.eta, w.beta, 21)
@@ -641,13 +641,13 @@ def test_step_captured_once_in_a_cuda_graph_and_replayed():
 
 
 @pytest.mark.parametrize("n_plain,n_replay", [(3, 2), (2, 2), (4, 4), (1, 1)])
-def test_reset_mask_of_the_last_reset_step_stays_readable_around_replay_mode(n_plain, n_replay):
+def test_reset_mask_of_the_last_reset_step_stays_readable_around_replay_mode(n_plain, n_replay, launch_path):
     """CSER_STATE_MASK_R is the reset mask of the last reset step that was executed - also when replay mode
     ends one step before a reset (its select kernel has then already prepared the next reset mask), when no
     reset ran during replay, and on the ordinary steps that follow."""
     d, n, bs, R1, R2, H = 4096 + 40, 4, 64, 4, 2, 3
     rng = np.random.default_rng(3)
-    opt = b.CSER(d, n, bs, R1, R2, H, 0.1, 0.9, 17, flags=b.FLAG_THREE_KERNELS)
+    opt = b.CSER(d, n, bs, R1, R2, H, 0.1, 0.9, 17)
     ref = CSEROracle(d, n, bs, R1, R2, H, 0.1, 0.9, 17, dtype=np.float32)
     x0 = rng.standard_normal(d).astype(np.float32)
     opt.set_x0(torch.from_numpy(x0).to(DEV)), ref.set_x0(x0)
