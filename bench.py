@@ -692,7 +692,7 @@ def main():
             "hbm_frac_of_8TBs": alg_bytes / (r["ms_per_step"] * 1e-3) / 1e9 / PEAK_NOMINAL_GBS,
             "algorithmic_bytes_per_step": alg_bytes,
             "roofline": r["roofline"], "cpu_baseline": cpu, "e2e": r["e2e"],
-            "gpu_launches": r["launches"], "clocks": r["clocks"],
+            "gpu_launches": r["launches"], "clocks": r["clocks"], "library": __graft_entry__.library_record(),
         }
         print(json.dumps(line))
     if world > 1:

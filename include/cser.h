@@ -362,6 +362,12 @@ int cser_step_noalloc(int64_t d, int32_t n_workers, int32_t block_size,
 /* Thread-local description of the last error in this thread ("" if none).  No passage of the paper: error reporting. */
 const char *cser_last_error(void);
 
+/*
+ * Identifier the build stamped into this binary (no passage of the paper: provenance): 16 hex digits
+ * over the library's sources and compiler flags, "unstamped" if it was built by other means.
+ */
+const char *cser_build_id(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -79,6 +79,8 @@ def lib():
     L.cser_debug_stall_next_staged_step.argtypes = [c.c_void_p, c.c_uint]
     L.cser_last_error.restype = c.c_char_p
     L.cser_last_error.argtypes = []
+    L.cser_build_id.restype = c.c_char_p
+    L.cser_build_id.argtypes = []
     for name in ("cser_set_x0", "cser_step", "cser_step_host", "cser_read_state", "cser_write_state",
                  "cser_debug_set_masks", "cser_grbs_mask", "cser_set_timing", "cser_last_kernel_ms"):
         getattr(L, name).restype = c.c_int
@@ -88,6 +90,10 @@ def lib():
 
 def cser_last_error():
     return lib().cser_last_error().decode()
+
+
+def cser_build_id():
+    return lib().cser_build_id().decode()
 
 
 def _check(rc, what):

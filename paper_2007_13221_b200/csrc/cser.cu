@@ -633,6 +633,11 @@ extern "C" {
 
 const char *cser_last_error(void) { return g_err; }
 
+#ifndef CSER_BUILD_ID
+#define CSER_BUILD_ID "unstamped"
+#endif
+const char *cser_build_id(void) { return CSER_BUILD_ID; }
+
 cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uint32_t R1,
                            uint32_t R2, int32_t H, float eta, float beta, uint64_t seed,
                            int64_t block_begin, uint32_t flags) {

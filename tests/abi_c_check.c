@@ -16,7 +16,7 @@ int main(void) {
         (fn_t)cser_launch_count, (fn_t)cser_last_error, (fn_t)cser_step_noalloc,
         (fn_t)cser_replay_begin, (fn_t)cser_step_replayable, (fn_t)cser_replay_end,
         (fn_t)cser_create_wshard, (fn_t)cser_wshard_message_elems,
-        (fn_t)cser_wshard_pack, (fn_t)cser_wshard_apply, (fn_t)cser_debug_stall_next_staged_step,
+        (fn_t)cser_wshard_pack, (fn_t)cser_wshard_apply, (fn_t)cser_debug_stall_next_staged_step, (fn_t)cser_build_id,
     };
     size_t i;
     for (i = 0; i < sizeof(fns) / sizeof(fns[0]); ++i)

@@ -53,6 +53,18 @@ def test_header_is_plain_c_and_the_library_links_from_c(tmp_path):
     assert declared <= used, declared - used
 
 
+def test_built_library_is_stamped_with_the_id_of_its_sources():
+    """build() stamps libcser.so with an id over its sources and flags and rebuilds when they differ, so a
+    stale binary cannot pass for a current one."""
+    import __graft_entry__
+    __graft_entry__.build()
+    from paper_2007_13221_b200 import binding
+    rec = __graft_entry__.library_record()
+    assert rec["matches_sources"] and len(rec["build_id"]) == 16, rec
+    assert binding.cser_build_id() == __graft_entry__.source_id(
+        os.path.join(ROOT, "paper_2007_13221_b200", "csrc", "cser.cu"))
+
+
 def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
     from paper_2007_13221_b200 import binding
     monkeypatch.setattr(binding, "_lib", None)
