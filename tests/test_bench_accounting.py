@@ -46,3 +46,33 @@ def test_overall_compression_ratio_matches_the_papers_formula_and_table():
         assert abs(replace(w, R1=R1, R2=R2, H=H).overall_ratio - overall) < 1e-9, (overall, R1, R2, H)
     assert abs(w.overall_ratio - 1.0 / (1 / 32 + 1 / 256)) < 1e-12
     assert replace(w, R1=0, R2=4, H=2).overall_ratio == 8.0            # CSER-PL: only the reset is exchanged
+
+
+def test_reference_arm_prints_the_contract_line_and_says_what_it_measured():
+    """`bench.py --impl reference` times the oracle on the host: one JSON line with the same metric, unit and
+    config object as the GPU arm's, `impl: reference`, a `cpu_baseline` describing the run, an `e2e` object
+    with no copies, and, when only a slab of the vector was timed, the measured slab and wall time beside the
+    extrapolated value."""
+    import json
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference", "--config", "1",
+                          "--steps", "2", "--warmup", "3"], capture_output=True, text=True, timeout=600,
+                         env={**os.environ, "CUDA_VISIBLE_DEVICES": ""})
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    w = synth.CONFIGS[1]
+    assert line["impl"] == "reference" and line["metric"] == bench.METRIC and line["unit"] == bench.UNIT
+    assert line["config"] == bench.config_of(w, 1)
+    assert line["higher_is_better"] is True and line["vs_baseline"] is None and line["steps"] == 2
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
+    # workload 1 runs real full-d steps: nothing is extrapolated, and value is the measured rate
+    assert line["extrapolated"] is False and line["measured_cols"] == w.d
+    assert abs(line["value"] - 1e3 / line["ms_per_step"]) < 1e-9 * line["value"] + 1e-12
+    # the larger workloads time a slab beyond the host caches and scale by columns
+    cols = bench.oracle_sample_cols(synth.CONFIGS[5])
+    assert cols % synth.CONFIGS[5].block_size == 0 and 8 * synth.CONFIGS[5].n_workers * cols >= 256 << 20
+    assert bench.oracle_sample_cols(synth.CONFIGS[1]) == w.d
