@@ -292,6 +292,9 @@ int cser_grbs_mask(uint64_t seed, uint64_t t, uint32_t which, int64_t block_begi
  *     sum msg over all ranks                (the caller's all-reduce, e.g. NCCL);
  *     cser_wshard_apply(h, msg, ...)        divide by n_total and finish the iteration.
  * Both PSyncs of a reset step (Algorithm 2 lines 6 and 11) share that one all-reduce.
+ * cser_wshard_pack returns with msg complete in stream order on `stream`, while the update of the
+ * unselected blocks still runs on a stream of the library's own: an all-reduce enqueued on
+ * `stream` right after the call overlaps it.  cser_wshard_apply (and cser_read_state) wait for it.
  * msg: device, fp32, at least cser_wshard_message_elems(h, reset_step) elements
  * (reset_step = whether the NEXT iteration t+1 is a multiple of H); a short last block is
  * padded with zeros.  grad: device fp32 [n_local, d].  With one rank holding all workers the

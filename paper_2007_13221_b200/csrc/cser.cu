@@ -98,6 +98,12 @@ struct cser_ctx {
     // ordered lists of the selected blocks, one set per mask buffer set (allocations of 2 B entries)
     uint32_t *pos_g = nullptr, *pos_r = nullptr, *olist_g = nullptr, *olist_r = nullptr;
     bool lists_ready[2] = {false, false};            // set k holds the lists of the masks in buffer set k
+    // Worker-sharded step: the streaming kernel runs on a side stream of its own and is joined only in
+    // cser_wshard_apply, so that the caller's all-reduce, enqueued on its stream right behind the pack
+    // kernel, overlaps the streaming of the unselected blocks.
+    cudaStream_t ws_side = nullptr;
+    cudaEvent_t ev_side = nullptr;
+    bool side_pending = false;
     bool wshard_open = false;                        // pack done, apply pending
     bool wshard_reset = false;
     // exact-count GRBS (CSER_FLAG_EXACT_COUNT)
@@ -769,6 +775,8 @@ cser_handle cser_create(int64_t d, int32_t n_workers, int32_t block_size, uint32
 void cser_destroy(cser_handle h) {
     if (!h) return;
     if (h->aux) cudaStreamSynchronize(h->aux);   // a select kernel may still be running ahead
+    if (h->ws_side) cudaStreamSynchronize(h->ws_side), cudaStreamDestroy(h->ws_side);
+    if (h->ev_side) cudaEventDestroy(h->ev_side);
     if (h->l2_persist) {
         cudaCtxResetPersistingL2Cache();
         cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, h->l2_limit_before);
@@ -907,6 +915,10 @@ int cser_read_state(cser_handle h, int which, void *dst, size_t dst_bytes, void 
     if (int rc = state_piece(h, which, &src, &bytes)) return rc;
     if (dst_bytes < bytes)
         return fail(CSER_ERR_TOO_SMALL, "cser_read_state: need %zu bytes, got %zu", bytes, dst_bytes);
+    if (h->side_pending) {      // worker-sharded step packed but not applied: its streaming kernel may still run
+        CU_TRY(cudaStreamWaitEvent((cudaStream_t)stream, h->ev_side, 0));
+        h->side_pending = false;
+    }
     if (h->replay && (which == CSER_STATE_MASK_G || which == CSER_STATE_MASK_R))
         src = which == CSER_STATE_MASK_G ? h->sb[0].mask_g : h->sb[0].mask_r;   // set 0 is the current one
     if (which == CSER_STATE_T) {
@@ -1015,6 +1027,8 @@ cser_handle cser_create_wshard(int64_t d, int32_t n_local, int32_t n_total, int3
     if (er == cudaSuccess) er = cudaMalloc(&h->pos_r, 2 * (size_t)h->B * sizeof(uint32_t));
     if (er == cudaSuccess) er = cudaMalloc(&h->olist_g, 2 * (size_t)h->B * sizeof(uint32_t));
     if (er == cudaSuccess) er = cudaMalloc(&h->olist_r, 2 * (size_t)h->B * sizeof(uint32_t));
+    if (er == cudaSuccess) er = cudaStreamCreateWithFlags(&h->ws_side, cudaStreamNonBlocking);
+    if (er == cudaSuccess) er = cudaEventCreateWithFlags(&h->ev_side, cudaEventDisableTiming);
     if (er != cudaSuccess) {
         fail(er == cudaErrorMemoryAllocation ? CSER_ERR_NOMEM : CSER_ERR_CUDA, "cser_create_wshard: %s",
              cudaGetErrorString(er));
@@ -1106,26 +1120,26 @@ int cser_wshard_pack(cser_handle h, const float *grad, float *msg, size_t msg_el
         if (int rc = launch_ordered_lists(h, h->cur, is_reset, h->t, s)) return abandon_iteration(h, t_before, rc);
     }
     h->lists_ready[h->cur] = false;          // consumed by this step
-    // the pack kernel (selected blocks) beside the streaming kernel (unselected blocks): disjoint columns
-    const bool beside = h->aux != nullptr;
-    cudaStream_t ps = s;
-    if (beside) {
-        CU_TRY(cudaEventRecord(h->ev_fork, s));
-        CU_TRY(cudaStreamWaitEvent(h->aux, h->ev_fork, 0));
-        ps = h->aux;
-    }
+    // Fork: the streaming kernel (unselected blocks) goes to the side stream, the next iteration's masks
+    // and ordered lists to the auxiliary stream; the pack kernel (selected blocks, disjoint columns) stays
+    // on the caller's stream, so the caller's all-reduce can start as soon as the message is complete.
+    CU_TRY(cudaEventRecord(h->ev_fork, s));
+    CU_TRY(cudaStreamWaitEvent(h->ws_side, h->ev_fork, 0));
     ShardParams P;
     bool v4;
     wshard_params(h, grad, msg, &v4, &P);
-    int rc = v4 ? launch_wshard<4>(h, P, is_reset, true, ps) : launch_wshard<1>(h, P, is_reset, true, ps);
-    if (!rc) rc = launch_step(h, grad, 0, h->d, is_reset, s, false);   // unselected blocks
-    if (beside) {
-        CU_TRY(cudaEventRecord(h->ev_join, h->aux));
-        CU_TRY(cudaStreamWaitEvent(s, h->ev_join, 0));
+    // the pack kernel first: it is small and the message is what the other ranks wait for
+    int rc = v4 ? launch_wshard<4>(h, P, is_reset, true, s) : launch_wshard<1>(h, P, is_reset, true, s);
+    if (!rc) rc = launch_step(h, grad, 0, h->d, is_reset, h->ws_side, false);
+    CU_TRY(cudaEventRecord(h->ev_side, h->ws_side));
+    h->side_pending = true;
+    if (rc) {
+        CU_TRY(cudaStreamWaitEvent(s, h->ev_side, 0));
+        h->side_pending = false;
+        return abandon_iteration(h, t_before, rc);
     }
-    if (rc) return abandon_iteration(h, t_before, rc);
-    if (beside && h->n_buf == 2) {
-        // the next iteration's masks and ordered lists, on the auxiliary stream behind the join
+    if (h->aux != nullptr && h->n_buf == 2) {
+        CU_TRY(cudaStreamWaitEvent(h->aux, h->ev_fork, 0));
         const uint64_t t_next = h->t + 1;
         const bool next_reset = (t_next % (uint64_t)h->H) == 0;
         const int nb = h->cur ^ 1;
@@ -1147,6 +1161,10 @@ int cser_wshard_apply(cser_handle h, const float *msg, void *stream) {
     if (h->n_total <= 0) return fail(CSER_ERR_INVALID, "cser_wshard_apply: not a worker-sharded handle");
     if (!h->wshard_open) return fail(CSER_ERR_INVALID, "cser_wshard_apply: no packed step pending");
     if (int rc = check_device_ptr(msg, "cser_wshard_apply: msg")) return rc;
+    if (h->side_pending) {      // the streaming kernel of this iteration
+        CU_TRY(cudaStreamWaitEvent((cudaStream_t)stream, h->ev_side, 0));
+        h->side_pending = false;
+    }
     ShardParams P;
     bool v4;
     wshard_params(h, nullptr, const_cast<float *>(msg), &v4, &P);
