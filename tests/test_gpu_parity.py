@@ -686,8 +686,8 @@ def test_random_shapes_parameters_and_flags_against_the_float32_oracle():
     then, host-gradient entry now and then): the state must equal the float32 oracle exactly."""
     rng = np.random.default_rng(20240607)
     for case in range(400):
-        n = int(rng.choice([1, 2, 3, 4, 5, 8, 9, 16, 17]))
-        bs = int(rng.choice([1, 3, 4, 8, 12, 16, 60, 64, 100, 128, 256]))
+        n = int(rng.choice([1, 2, 3, 4, 5, 8, 9, 16, 17, 33]))
+        bs = int(rng.choice([1, 3, 4, 8, 12, 16, 60, 64, 100, 128, 256, 1024]))
         d = int(rng.integers(1, 40)) * bs + int(rng.integers(0, bs)) if rng.random() < 0.7 else int(rng.integers(1, 3000))
         R1 = int(rng.choice([0, 1, 2, 3, 4, 7, 32]))
         R2 = int(rng.choice([1, 2, 3, 4, 16]))
@@ -699,6 +699,7 @@ def test_random_shapes_parameters_and_flags_against_the_float32_oracle():
         seed = int(rng.integers(0, 2**62))
         flags = (b.FLAG_NO_ERROR_ARRAY if impl2 else 0) | (b.FLAG_EXACT_COUNT if exact else 0)
         flags |= b.FLAG_THREE_KERNELS if rng.random() < 0.4 else 0
+        flags |= b.FLAG_STAGED_SELECTED if rng.random() < 0.3 else 0     # (implies the three kernels)
         opt = b.CSER(d, n, bs, R1, R2, H, eta, beta, seed, flags=flags)
         ref = (CSERImpl2Oracle if impl2 else CSEROracle)(d, n, bs, R1, R2, H, eta, beta, seed, dtype=np.float32,
                                                          exact_count=exact)
