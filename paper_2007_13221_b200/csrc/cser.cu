@@ -634,6 +634,14 @@ bool begin_iteration(cser_ctx *h) {
 
 }  // namespace
 
+namespace {
+// Handles with CSER_FLAG_L2_RESIDENT share one limit of the CUDA context (the L2 set-aside): it is raised by
+// whoever needs more and put back, with the persisting lines released, only when the last such handle of
+// the device is destroyed.
+int g_l2_users[64] = {};
+size_t g_l2_limit_before[64] = {};
+}  // namespace
+
 // ------------------------------------------------------------------ C ABI
 extern "C" {
 
@@ -715,9 +723,15 @@ cser_handle cser_create_ex(int64_t d, int32_t n_workers, int32_t block_size, uin
         if (h->state_bytes <= (size_t)max_persist && h->state_bytes <= (size_t)max_window) {
             size_t cur_limit = 0;
             if (cudaDeviceGetLimit(&cur_limit, cudaLimitPersistingL2CacheSize) == cudaSuccess) {
-                h->l2_limit_before = cur_limit;
+                const bool slot = h->device >= 0 && h->device < 64;
+                const bool first = !slot || g_l2_users[h->device] == 0;
+                h->l2_limit_before = first ? cur_limit : (slot ? g_l2_limit_before[h->device] : cur_limit);
                 const size_t want = cur_limit > h->state_bytes ? cur_limit : h->state_bytes;
                 h->l2_persist = cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want) == cudaSuccess;
+                if (h->l2_persist && slot) {
+                    if (first) g_l2_limit_before[h->device] = cur_limit;
+                    g_l2_users[h->device]++;
+                }
             }
             cudaGetLastError();
         }
@@ -778,9 +792,12 @@ void cser_destroy(cser_handle h) {
     if (h->ws_side) cudaStreamSynchronize(h->ws_side), cudaStreamDestroy(h->ws_side);
     if (h->ev_side) cudaEventDestroy(h->ev_side);
     if (h->l2_persist) {
-        cudaCtxResetPersistingL2Cache();
-        cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, h->l2_limit_before);
-        cudaGetLastError();
+        const bool slot = h->device >= 0 && h->device < 64;
+        if (!slot || --g_l2_users[h->device] == 0) {      // the last L2-resident handle of this device
+            cudaCtxResetPersistingL2Cache();
+            cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, h->l2_limit_before);
+            cudaGetLastError();
+        }
     }
     cudaFree(h->state_base);
     cudaFree(h->sb[0].mask_g), cudaFree(h->sb[0].mask_r), cudaFree(h->sb[0].list);

@@ -547,7 +547,18 @@ def test_l2_resident_state_gives_the_same_results(launch_path):
     big.step(torch.zeros((8, 30_000_000), device=DEV))
     for which in (b.STATE_X, b.STATE_E):
         assert torch.equal(a.state(which), c.state(which))
-    a.close(), c.close(), big.close()
+    # two L2-resident handles share the context's set-aside: destroying one leaves the other's in place
+    c2 = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, 3, flags=b.FLAG_L2_RESIDENT)
+    c2.set_x0(x0)
+    c.close()
+    a2 = b.CSER(w.d, w.n_workers, w.block_size, w.R1, w.R2, w.H, w.eta, w.beta, 3)
+    a2.set_x0(x0)
+    for t in range(1, 6):
+        g = synth.gradients(w, t, DEV)
+        a2.step(g), c2.step(g)
+    for which in (b.STATE_X, b.STATE_E):
+        assert torch.equal(a2.state(which), c2.state(which))
+    a.close(), a2.close(), c2.close(), big.close()
 
 
 def test_misaligned_gradient_pointer_takes_the_scalar_path():
