@@ -218,8 +218,11 @@ def _cols_of(blocks, w):
     return np.concatenate(parts)
 
 
-def _full_size_parity(cfg, steps=None, n_random=192, impl2=False, flags=0):
+def _full_size_parity(cfg, steps=None, n_random=192, impl2=False, flags=0, ratios=None):
     w = synth.CONFIGS[cfg]
+    if ratios is not None:                      # same shape, other (R1, R2, H)
+        from dataclasses import replace
+        w = replace(w, R1=ratios[0], R2=ratios[1], H=ratios[2])
     oracle = CSERImpl2Oracle if impl2 else CSEROracle
     steps = w.steps if steps is None else steps
     rng = np.random.default_rng(cfg)
@@ -321,6 +324,14 @@ def test_config1_full_vector_every_element(launch_path):
 @pytest.mark.parametrize("cfg", [2, 3, 4])
 def test_full_size_configs_on_sampled_blocks(cfg):
     _full_size_parity(cfg)
+
+
+@pytest.mark.parametrize("cfg,ratios", [(2, (4, 4, 2)), (5, (4, 8, 2))])
+def test_full_size_shapes_with_many_selected_blocks_on_sampled_blocks(cfg, ratios):
+    """The WRN-sized and the BERT-large-sized vector with a quarter of the blocks selected: every iteration
+    goes through the single-launch kernel (the per-iteration rule), at full size, past 2^31 elements for the
+    larger one; sampled whole blocks against the oracle, Lemma 1 and e = 0 after resets on the whole state."""
+    _full_size_parity(cfg, steps=6, n_random=96, ratios=ratios)
 
 
 def test_config5_bert_large_sized_on_sampled_blocks():
