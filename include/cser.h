@@ -156,10 +156,10 @@ cser_handle cser_create_slab(int64_t d, int32_t n_workers, int32_t block_size,
  *       (same Philox draws, same arithmetic, bit-identical results), in two cases: when the iteration
  *       moves at most 256 MB (n_workers * d * 28 bytes with momentum and an error array), because it
  *       would take a few tens of microseconds and the kernel boundaries would cost as much as the
- *       traffic; and, with at most 8 workers, when a large share of the blocks is selected in that
- *       iteration (1/R1 >= 1/4 on an ordinary step, 1/R1 + 1/R2 >= 1/10 on a reset step), because walking
- *       all columns in their natural order then beats sending scattered blocks through the selected-block
- *       kernel.  This flag keeps the three kernels for every iteration.  Steps with injected masks,
+ *       traffic; and when a large share of the blocks is selected in that iteration (with up to 8
+ *       workers: 1/R1 >= 1/4 on an ordinary step, 1/R1 + 1/R2 >= 1/10 on a reset step; with 9 to 16
+ *       workers: R1 = 1, or 1/R1 + 1/R2 >= 1/5 on a reset step), because walking all columns in their
+ *       natural order then beats sending scattered blocks through the selected-block kernel.  This flag keeps the three kernels for every iteration.  Steps with injected masks,
  *       exact-count masks, replayable steps, cser_step_host and vectors whose d or block_size is not a
  *       multiple of 4 use the three kernels in any case.
  */

@@ -253,23 +253,28 @@ long long step_bytes_bound(const cser_ctx *h) {
 // WRN-40-8-sized vector (n = 8; ordinary / reset steps in ms, three kernels against one launch): R = 2
 // 1.113 / 1.526 against 1.077 / 1.179; R = 4 1.165 / 1.449 against 1.164 / 1.196; R = 8 1.179 / 1.338
 // against 1.206 / 1.219; R = 16 1.177 / 1.256 against 1.226 / 1.233; R = 32 1.178 / 1.226 against
-// 1.237 / 1.242.  Hence one launch from a selected share of 1/4 on ordinary steps and of 1/10 on reset
-// steps (update mask and reset mask together), for up to 8 workers (with 16 the walk over all
-// columns loses more than it gains).
-#ifndef CSER_FUSED_SHARE_PLAIN
-#define CSER_FUSED_SHARE_PLAIN 0.25
-#define CSER_FUSED_SHARE_RESET 0.10
-#define CSER_FUSED_SHARE_MAX_WORKERS 8
-#endif
+// 1.237 / 1.242.  Hence, for up to 8 workers, one launch from a selected share of 1/4 on ordinary steps
+// and of 1/10 on reset steps (update mask and reset mask together).  With 16 workers (ResNet-50-sized
+// vector, block 1024) the walk over all columns pays later: ordinary steps only when everything is
+// selected (R = 2: 1.554 against 1.566 ms, R = 4: 1.628 against 1.716), reset steps from a share of 1/5
+// (R = 8: 1.832 against 1.806, R = 4: 1.941 against 1.771, R = 2: 2.015 against 1.732).  Beyond 16
+// workers nothing was measured and the three kernels are kept.
+struct FusedShare { double plain, reset; };
+FusedShare fused_share_thresholds(int n) {
+    if (n <= 8) return {0.25, 0.10};
+    if (n <= 16) return {1.0, 0.20};
+    return {2.0, 2.0};      // never
+}
 // Whether iteration number t of handle h goes through the single-launch kernel (given a gradient
 // pointer that allows 128-bit loads).
 bool fused_for_iteration(const cser_ctx *h, uint64_t t) {
     if (!(h->fused_small && h->vec4 && !h->exact && !h->replay && h->n_total == 0 && h->n_buf == 2)) return false;
     if (step_bytes_bound(h) <= kFusedMaxBytes) return true;
-    if (h->n > CSER_FUSED_SHARE_MAX_WORKERS || h->d / 4 > 0xffffffffll) return false;
+    if (h->d / 4 > 0xffffffffll) return false;
     const bool is_reset = (t % (uint64_t)h->H) == 0;
     const double share = (h->R1 ? 1.0 / h->R1 : 0.0) + (is_reset ? 1.0 / h->R2 : 0.0);
-    return share >= (is_reset ? CSER_FUSED_SHARE_RESET : CSER_FUSED_SHARE_PLAIN);
+    const FusedShare th = fused_share_thresholds(h->n);
+    return share >= (is_reset ? th.reset : th.plain);
 }
 
 // Work-unit geometry of the staged selected-block kernel: C vector columns per unit so that all n
