@@ -385,9 +385,13 @@ def run_workload(w, K, W, dev, rank, world, ring_n=0, with_e2e=True, flush_l2=Fa
     # end to end: gradients start in pinned host memory every step; a result is read back
     out["e2e"] = None
     if with_e2e:
-        host_ring = [torch.empty((w.n_workers, w.d), dtype=torch.float32).pin_memory() for _ in range(2)]
+        # two pinned host buffers, alternated; one when a buffer is several GB (every rank pins its own)
+        host_ring = [torch.empty((w.n_workers, w.d), dtype=torch.float32).pin_memory()
+                     for _ in range(1 if g_bytes > 4e9 else 2)]
         for hb, gb in zip(host_ring, ring):
             hb.copy_(gb)
+        if len(host_ring) == 1:
+            host_ring.append(host_ring[0])
         mask_host = torch.empty(w.n_blocks, dtype=torch.uint8).pin_memory()
         ke = max(3, min(K, 12))
         for k in range(2):
